@@ -1,0 +1,191 @@
+/*
+ * chiron_kv.h -- C ABI of the decode-iteration hot path: paged grouped-query decode attention
+ * over a bf16 KV cache, and the paged KV append of each iteration's new token.
+ *
+ * Framing (paper): a serving instance runs a continuous batch of requests (Section 2.1,
+ * "Continuous Batching"); every decode iteration generates one token per running request from
+ * the keys and values of all its previous tokens, which are kept in the KV cache ("Inference
+ * Primer"); the cache is managed in pages allocated on demand ("PagedAttention").  The
+ * iteration's latency as a function of batch size is the quantity the local autoscaler weighs
+ * against the inter-token-latency SLO (Section 4.1 "Local Backpressure", Algorithm 1).
+ *
+ * Conventions
+ *  - All functions are extern "C", return an int32 status (CKV_OK or a negative CKV_E* code) and
+ *    never throw.  ckv_last_error() gives a message for the calling thread's last failure.
+ *  - "d_" pointers are DEVICE pointers, "h_" pointers are HOST pointers.  Every device buffer is
+ *    owned by the caller; the library never allocates or frees device memory.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls only enqueue
+ *    work on it and return without synchronising unless stated otherwise.
+ *  - bf16 values are raw 16-bit patterns (upper half of an IEEE binary32).
+ *  - KV pool layout:  bf16 pool[num_layers][num_pages][num_kv_heads][2 (0=K,1=V)][page_size][head_dim]
+ *    so the K and V rows of one (page, KV head) form one contiguous block.
+ *  - Block tables: int32 [batch][max_pages_per_req]; entry i of row r is the physical page that
+ *    holds tokens [i*page_size, (i+1)*page_size) of request r.  Only the first
+ *    ceil(seq_lens[r]/page_size) entries of a row are read.  Requests may share pages for
+ *    reading; append targets must be distinct.
+ *  - seq_lens[r] is the context length AFTER this iteration's append: attention of request r
+ *    covers tokens 0 .. seq_lens[r]-1 and the appended token has position seq_lens[r]-1.
+ *  - Query head h uses KV head h / (num_q_heads / num_kv_heads).  Softmax scale is
+ *    1/sqrt(head_dim).
+ *  - Invalid device-side data (a length < 1 or beyond the table, a page id outside the pool) is
+ *    never followed: the access is skipped or redirected to page 0, a bit is set in a device
+ *    status word, and kv_check_status() reports it.  Output rows of a request with an invalid
+ *    length are zero-filled; rows of a request with an invalid page id are unspecified.
+ *
+ * Supported shapes: head_dim 64 or 128, page_size 16, 1 <= num_q_heads/num_kv_heads <= 8.
+ */
+#ifndef CHIRON_KV_H
+#define CHIRON_KV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define CKV_OK        0
+#define CKV_EINVAL   (-1)   /* bad argument or unsupported shape */
+#define CKV_ENOMEM   (-2)   /* a caller-provided buffer is too small */
+#define CKV_ECUDA    (-3)   /* a CUDA runtime/driver call failed (see ckv_last_error) */
+#define CKV_EBOUNDS  (-4)   /* device saw an out-of-range length or page id */
+#define CKV_ETIMEOUT (-5)   /* a bounded device-side wait gave up */
+
+/* bits of the device status word */
+#define CKV_STATUS_BAD_LENGTH 1u
+#define CKV_STATUS_BAD_PAGE   2u
+#define CKV_STATUS_WAIT_LIMIT 4u
+
+typedef struct ckv_config {
+    int32_t num_layers;         /* layers sharing block tables, each with its own pool slice */
+    int32_t num_q_heads;        /* Hq */
+    int32_t num_kv_heads;       /* Hkv, divides Hq */
+    int32_t head_dim;           /* d: 64 or 128 */
+    int32_t page_size;          /* P: 16 */
+    int32_t num_pages;          /* physical pages per layer */
+    int32_t max_pages_per_req;  /* row width of the block tables */
+    int32_t max_batch;          /* largest batch any call will pass */
+} ckv_config;
+
+typedef struct ckv_pool ckv_pool;   /* host-side handle; holds no device allocations of its own */
+
+/* Bytes of the KV pool for this configuration (0 if the configuration is invalid). */
+size_t kv_pool_bytes(const ckv_config *cfg);
+
+/* Bytes of scratch the library needs: status word, split-KV plan, partial results, and staging
+ * for decode_step_host (0 if the configuration is invalid). */
+size_t kv_workspace_bytes(const ckv_config *cfg);
+
+/*
+ * Create the host-side handle for a pool that lives in caller-owned device memory (the paged
+ * KV cache of Section 2.1 "PagedAttention").  d_pool must be 1024-byte aligned and hold
+ * kv_pool_bytes(); d_workspace must be 256-byte aligned and hold kv_workspace_bytes().  The
+ * workspace is cleared on the default stream and the call synchronises once.  `device` is the
+ * CUDA device ordinal both buffers live on.  Errors: CKV_EINVAL (shape, alignment),
+ * CKV_ENOMEM (a size too small), CKV_ECUDA.
+ */
+int32_t kv_pool_create(const ckv_config *cfg, void *d_pool, size_t pool_bytes,
+                       void *d_workspace, size_t workspace_bytes, int32_t device,
+                       ckv_pool **out_pool);
+
+/* Free the host handle (synchronises the device first).  Device memory stays with the caller. */
+int32_t kv_pool_destroy(ckv_pool *pool);
+
+/*
+ * KV append (Section 2.1 "Inference Primer": the key and value vectors of generated tokens are
+ * cached for later tokens).  For each request r < batch and KV head kh, copies bit-exactly
+ *   d_k_new[r][kh][:] -> pool[layer][page][kh][K][slot][:]   and   d_v_new -> ...[V]...
+ * with page = d_block_tables[r][(seq_lens[r]-1)/P], slot = (seq_lens[r]-1) % P.
+ * d_k_new, d_v_new: bf16 [batch][num_kv_heads][head_dim], 16-byte aligned.  No other byte of
+ * the pool is written.  Errors: CKV_EINVAL (layer/batch out of range, NULL), CKV_ECUDA.
+ */
+int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch,
+                  const int32_t *d_block_tables, const int32_t *d_seq_lens,
+                  const void *d_k_new, const void *d_v_new, void *stream);
+
+/*
+ * Decode attention for one layer of the running batch (the "self-attention computation" whose
+ * cost grows with batch size, Section 2.3 "Motivation and Characterization" and Section 4.1):
+ *   out[r][h][:] = sum_j softmax_j( q[r][h].k_j / sqrt(d) ) v_j ,  j over request r's context,
+ * computed as split-KV partials over balanced page ranges followed by a log-sum-exp combine.
+ * d_q, d_out: bf16 [batch][num_q_heads][head_dim], 16-byte aligned; every row of d_out is
+ * overwritten.  Enqueues a plan kernel, the attention kernel and the combine kernel.
+ * Errors: CKV_EINVAL, CKV_ECUDA.
+ */
+int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch,
+                         const int32_t *d_block_tables, const int32_t *d_seq_lens,
+                         const void *d_q, void *d_out, void *stream);
+
+/*
+ * The split-KV partition the next decode_attention would use for these lengths, copied to the
+ * host for inspection (synchronises `stream`).  A "tile" is 64 consecutive tokens of one
+ * (request, KV head); tiles are numbered request-major, then KV head, then position, and CTA c
+ * owns tiles [c*tiles_per_cta, min((c+1)*tiles_per_cta, total_tiles)).
+ *   h_header[4]   : total_tiles, tiles_per_cta, num_ctas (launched), num_ctas_with_work
+ *   h_cta_start   : int32 [num_ctas][4] = request, kv head, first tile within that
+ *                   (request, kv head), global index of the CTA's first tile; -1s if idle
+ * h_cta_start must hold 4*ckv_get_partition() ints.  Errors: CKV_EINVAL, CKV_ECUDA.
+ */
+int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *stream,
+                    int32_t *h_header, int32_t *h_cta_start);
+
+/* Number of CTAs the partition is balanced over (default: one per SM).  Setting it changes
+ * only how the context is split, never the result beyond fp32 summation order.
+ * 1 <= num_ctas <= 1024.  Errors: CKV_EINVAL. */
+int32_t ckv_set_partition(ckv_pool *pool, int32_t num_ctas);
+int32_t ckv_get_partition(const ckv_pool *pool);
+
+/* Synchronise `stream`, read and clear the device status word.  Returns CKV_OK, CKV_EBOUNDS
+ * (bad length or page id seen), CKV_ETIMEOUT, or CKV_ECUDA.  *out_bits (may be NULL) receives
+ * the raw CKV_STATUS_* bits. */
+int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits);
+
+/*
+ * One whole iteration for one layer with HOST buffers (pinned memory recommended): copies the
+ * tables, lengths, q, k_new and v_new to the device, runs kv_append and decode_attention, copies
+ * the output back and synchronises `stream`.  h_out: bf16 [batch][num_q_heads][head_dim].
+ * Errors: as kv_append / decode_attention.
+ */
+int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch,
+                         const int32_t *h_block_tables, const int32_t *h_seq_lens,
+                         const void *h_q, const void *h_k_new, const void *h_v_new,
+                         void *h_out, void *stream);
+
+/*
+ * Iteration latency against batch size: the curve Algorithm 1 reads as ITL(batch size)
+ * (Section 2.1, figure "Variation in inter-token latency and token throughput with
+ * increasing batch size"; Section 4.1).  For each i < n_sizes, runs `warmup` untimed and `iters` timed
+ * steps on the first batch_sizes[i] requests of the given arrays; a step is kv_append +
+ * decode_attention for every layer.  Per-layer inputs are laid out
+ *   d_q, d_out [num_layers][batch_stride][Hq][d],  d_k_new, d_v_new [num_layers][batch_stride][Hkv][d].
+ * Each timed step is bracketed by CUDA events on `stream`; if d_flush is not NULL,
+ * flush_bytes of it are overwritten before every step (outside the timed bracket) so that no
+ * step starts with its inputs in L2.  Synchronises.  out_median_us / out_min_us: [n_sizes].
+ * Errors: CKV_EINVAL, CKV_ECUDA, CKV_EBOUNDS/CKV_ETIMEOUT if the status word is set afterwards.
+ */
+int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch_sizes,
+                           int32_t batch_stride,
+                           const int32_t *d_block_tables, const int32_t *d_seq_lens,
+                           const void *d_q, const void *d_k_new, const void *d_v_new, void *d_out,
+                           int32_t warmup, int32_t iters, void *d_flush, size_t flush_bytes,
+                           void *stream, double *out_median_us, double *out_min_us);
+
+/*
+ * Per-kernel timing for roofline accounting: while enabled, decode_attention brackets its
+ * attention kernel with CUDA events on the launch stream (up to 4096 launches are kept).
+ * ckv_profile_read synchronises the device and returns the summed kernel time and the number
+ * of launches since enabling.  Errors: CKV_EINVAL, CKV_ECUDA.
+ */
+int32_t ckv_profile_enable(ckv_pool *pool, int32_t enable);
+int32_t ckv_profile_read(ckv_pool *pool, double *out_attention_ms, int32_t *out_launches);
+
+/* Kernels launched through this handle since creation (append, plan, attention, combine). */
+int64_t ckv_launch_count(const ckv_pool *pool);
+
+/* Message describing the calling thread's most recent failure ("" if none). */
+const char *ckv_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CHIRON_KV_H */

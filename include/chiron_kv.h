@@ -78,7 +78,7 @@ size_t kv_workspace_bytes(const ckv_config *cfg);
 
 /*
  * Create the host-side handle for a pool that lives in caller-owned device memory (the paged
- * KV cache of Section 2.1 "PagedAttention").  d_pool must be 1024-byte aligned and hold
+ * KV cache of Section 2.1 "PagedAttention").  d_pool must be 256-byte aligned and hold
  * kv_pool_bytes(); d_workspace must be 256-byte aligned and hold kv_workspace_bytes().  The
  * workspace is cleared on the default stream and the call synchronises once.  `device` is the
  * CUDA device ordinal both buffers live on.  Errors: CKV_EINVAL (shape, alignment),

@@ -1,0 +1,229 @@
+"""ctypes binding of libchiron_kv.so (see include/chiron_kv.h): argument marshalling only.
+
+Every computation runs in the library's CUDA kernels.  There is no fallback: if the shared
+library has not been built, importing this module raises.  torch is used for device memory and
+streams, nothing else.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIBRARY = os.path.join(_HERE, "libchiron_kv.so")
+
+CKV_OK, CKV_EINVAL, CKV_ENOMEM, CKV_ECUDA, CKV_EBOUNDS, CKV_ETIMEOUT = 0, -1, -2, -3, -4, -5
+STATUS_BAD_LENGTH, STATUS_BAD_PAGE, STATUS_WAIT_LIMIT = 1, 2, 4
+
+EXPORTS = (
+    "kv_pool_bytes", "kv_workspace_bytes", "kv_pool_create", "kv_pool_destroy", "kv_append",
+    "decode_attention", "decode_plan", "ckv_set_partition", "ckv_get_partition", "kv_check_status",
+    "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
+    "ckv_launch_count", "ckv_last_error",
+)
+
+
+class CkvError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__("chiron_kv error %d: %s" % (code, message))
+        self.code = code
+
+
+class Config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in (
+        "num_layers", "num_q_heads", "num_kv_heads", "head_dim", "page_size", "num_pages",
+        "max_pages_per_req", "max_batch")]
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIBRARY):
+        raise ImportError(
+            "libchiron_kv.so is missing at %s: build it with `python -m paper_2501_08090_b200.build` "
+            "(nvcc, sm_100a).  There is no CPU fallback." % LIBRARY)
+    lib = ctypes.CDLL(LIBRARY)
+    i32, i64, vp, sz = ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p, ctypes.c_size_t
+    cfgp = ctypes.POINTER(Config)
+    lib.kv_pool_bytes.restype = sz; lib.kv_pool_bytes.argtypes = [cfgp]
+    lib.kv_workspace_bytes.restype = sz; lib.kv_workspace_bytes.argtypes = [cfgp]
+    lib.kv_pool_create.restype = i32
+    lib.kv_pool_create.argtypes = [cfgp, vp, sz, vp, sz, i32, ctypes.POINTER(vp)]
+    lib.kv_pool_destroy.restype = i32; lib.kv_pool_destroy.argtypes = [vp]
+    lib.kv_append.restype = i32; lib.kv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.decode_attention.restype = i32; lib.decode_attention.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.decode_plan.restype = i32; lib.decode_plan.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.ckv_set_partition.restype = i32; lib.ckv_set_partition.argtypes = [vp, i32]
+    lib.ckv_get_partition.restype = i32; lib.ckv_get_partition.argtypes = [vp]
+    lib.kv_check_status.restype = i32; lib.kv_check_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.decode_step_host.restype = i32; lib.decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.step_latency_sweep.restype = i32
+    lib.step_latency_sweep.argtypes = [vp, i32, vp, i32, vp, vp, vp, vp, vp, vp, i32, i32, vp, sz, vp, vp, vp]
+    lib.ckv_profile_enable.restype = i32; lib.ckv_profile_enable.argtypes = [vp, i32]
+    lib.ckv_profile_read.restype = i32
+    lib.ckv_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
+    lib.ckv_launch_count.restype = i64; lib.ckv_launch_count.argtypes = [vp]
+    lib.ckv_last_error.restype = ctypes.c_char_p; lib.ckv_last_error.argtypes = []
+    return lib
+
+
+lib = _load()
+
+
+def last_error() -> str:
+    return lib.ckv_last_error().decode("utf-8", "replace")
+
+
+def _check(rc: int) -> None:
+    if rc != CKV_OK:
+        raise CkvError(rc, last_error())
+
+
+def make_config(num_layers, num_q_heads, num_kv_heads, head_dim, num_pages, max_pages_per_req,
+                max_batch, page_size=16) -> Config:
+    return Config(num_layers, num_q_heads, num_kv_heads, head_dim, page_size, num_pages,
+                  max_pages_per_req, max_batch)
+
+
+def kv_pool_bytes(cfg: Config) -> int:
+    return int(lib.kv_pool_bytes(ctypes.byref(cfg)))
+
+
+def kv_workspace_bytes(cfg: Config) -> int:
+    return int(lib.kv_workspace_bytes(ctypes.byref(cfg)))
+
+
+def _dev_ptr(t: Optional[torch.Tensor], dtype=None) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda or not t.is_contiguous():
+        raise ValueError("expected a contiguous CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError("expected dtype %s, got %s" % (dtype, t.dtype))
+    return t.data_ptr()
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    return (stream or torch.cuda.current_stream()).cuda_stream
+
+
+class KvPool:
+    """A paged bf16 KV cache in caller-owned device memory plus the library's scratch.
+
+    `pool` (bf16, kv_pool_bytes) and `workspace` (uint8, kv_workspace_bytes) may be passed in;
+    otherwise they are allocated with torch on `device`.  The tensors are kept alive here.
+    """
+
+    def __init__(self, cfg: Config, device="cuda:0", pool: Optional[torch.Tensor] = None,
+                 workspace: Optional[torch.Tensor] = None):
+        self.cfg = cfg
+        self.device = torch.device(device)
+        need_pool, need_ws = kv_pool_bytes(cfg), kv_workspace_bytes(cfg)
+        if need_pool == 0 or need_ws == 0:
+            raise CkvError(CKV_EINVAL, last_error())
+        if pool is None:
+            pool = torch.empty(need_pool // 2, dtype=torch.bfloat16, device=self.device)
+        if workspace is None:
+            workspace = torch.empty(need_ws, dtype=torch.uint8, device=self.device)
+        self.pool, self.workspace = pool, workspace
+        self._h = ctypes.c_void_p()
+        index = self.device.index if self.device.index is not None else torch.cuda.current_device()
+        _check(lib.kv_pool_create(ctypes.byref(cfg), _dev_ptr(pool), pool.numel() * pool.element_size(),
+                                  _dev_ptr(workspace), workspace.numel() * workspace.element_size(),
+                                  index, ctypes.byref(self._h)))
+
+    # -- lifetime
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None and self._h.value:
+            lib.kv_pool_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def pool_view(self) -> torch.Tensor:
+        """[layers][pages][Hkv][2][P][d] view of the pool tensor."""
+        c = self.cfg
+        n = c.num_layers * c.num_pages * c.num_kv_heads * 2 * c.page_size * c.head_dim
+        return self.pool.view(-1)[:n].view(c.num_layers, c.num_pages, c.num_kv_heads, 2, c.page_size, c.head_dim)
+
+    # -- the hot path
+    def kv_append(self, layer: int, block_tables, seq_lens, k_new, v_new, stream=None) -> None:
+        batch = int(seq_lens.shape[0])
+        _check(lib.kv_append(self._h, layer, batch, _dev_ptr(block_tables, torch.int32),
+                             _dev_ptr(seq_lens, torch.int32), _dev_ptr(k_new, torch.bfloat16),
+                             _dev_ptr(v_new, torch.bfloat16), _stream_ptr(stream)))
+
+    def decode_attention(self, layer: int, block_tables, seq_lens, q, out, stream=None) -> None:
+        batch = int(seq_lens.shape[0])
+        _check(lib.decode_attention(self._h, layer, batch, _dev_ptr(block_tables, torch.int32),
+                                    _dev_ptr(seq_lens, torch.int32), _dev_ptr(q, torch.bfloat16),
+                                    _dev_ptr(out, torch.bfloat16), _stream_ptr(stream)))
+
+    def decode_plan(self, seq_lens, stream=None):
+        """(header dict, int32 [num_ctas][4] array of span starts)."""
+        batch = int(seq_lens.shape[0])
+        header = np.zeros(4, dtype=np.int32)
+        starts = np.zeros((self.get_partition(), 4), dtype=np.int32)
+        _check(lib.decode_plan(self._h, batch, _dev_ptr(seq_lens, torch.int32), _stream_ptr(stream),
+                               header.ctypes.data, starts.ctypes.data))
+        keys = ("total_tiles", "tiles_per_cta", "num_ctas", "ctas_with_work")
+        return dict(zip(keys, header.tolist())), starts
+
+    def set_partition(self, num_ctas: int) -> None:
+        _check(lib.ckv_set_partition(self._h, int(num_ctas)))
+
+    def get_partition(self) -> int:
+        return int(lib.ckv_get_partition(self._h))
+
+    def check_status(self, stream=None, raise_on_error: bool = True) -> int:
+        bits = ctypes.c_uint32(0)
+        rc = lib.kv_check_status(self._h, _stream_ptr(stream), ctypes.byref(bits))
+        if rc != CKV_OK and raise_on_error:
+            raise CkvError(rc, last_error())
+        return int(bits.value)
+
+    def decode_step_host(self, layer: int, block_tables, seq_lens, q, k_new, v_new, out, stream=None) -> None:
+        """Host (CPU, ideally pinned) tensors in, host tensor out; synchronises."""
+        for t in (block_tables, seq_lens, q, k_new, v_new, out):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("decode_step_host takes contiguous host tensors")
+        batch = int(seq_lens.shape[0])
+        _check(lib.decode_step_host(self._h, layer, batch, block_tables.data_ptr(), seq_lens.data_ptr(),
+                                    q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
+                                    _stream_ptr(stream)))
+
+    def step_latency_sweep(self, batch_sizes: Sequence[int], block_tables, seq_lens, q, k_new, v_new, out,
+                           warmup: int = 3, iters: int = 20, flush: Optional[torch.Tensor] = None,
+                           stream=None):
+        """Median and minimum microseconds per step for each batch size (numpy float64 arrays)."""
+        sizes = np.asarray(list(batch_sizes), dtype=np.int32)
+        med = np.zeros(sizes.size, dtype=np.float64)
+        mn = np.zeros(sizes.size, dtype=np.float64)
+        stride = int(seq_lens.shape[0])
+        fl_ptr = _dev_ptr(flush) if flush is not None else None
+        fl_bytes = flush.numel() * flush.element_size() if flush is not None else 0
+        _check(lib.step_latency_sweep(self._h, int(sizes.size), sizes.ctypes.data, stride,
+                                      _dev_ptr(block_tables, torch.int32), _dev_ptr(seq_lens, torch.int32),
+                                      _dev_ptr(q, torch.bfloat16), _dev_ptr(k_new, torch.bfloat16),
+                                      _dev_ptr(v_new, torch.bfloat16), _dev_ptr(out, torch.bfloat16),
+                                      int(warmup), int(iters), fl_ptr, fl_bytes, _stream_ptr(stream),
+                                      med.ctypes.data, mn.ctypes.data))
+        return med, mn
+
+    def profile_enable(self, enable: bool) -> None:
+        _check(lib.ckv_profile_enable(self._h, 1 if enable else 0))
+
+    def profile_read(self):
+        ms = ctypes.c_double(0.0)
+        n = ctypes.c_int32(0)
+        _check(lib.ckv_profile_read(self._h, ctypes.byref(ms), ctypes.byref(n)))
+        return float(ms.value), int(n.value)
+
+    def launch_count(self) -> int:
+        return int(lib.ckv_launch_count(self._h))

@@ -1,0 +1,513 @@
+// Host runtime and C ABI (include/chiron_kv.h) of the paged decode-attention library.
+// Argument checking, workspace carving, tensor-map creation, kernel launches and timing loops.
+// No device memory is allocated here: pool and workspace belong to the caller.
+#include "chiron_kv.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "ckv_device.cuh"
+
+namespace {
+
+thread_local char g_error[512] = "";
+
+int32_t fail(int32_t code, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof g_error, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define CKV_CUDA(call)                                                                        \
+    do {                                                                                      \
+        cudaError_t e_ = (call);                                                              \
+        if (e_ != cudaSuccess)                                                                \
+            return fail(CKV_ECUDA, "%s failed: %s (%s:%d)", #call, cudaGetErrorString(e_),    \
+                        __FILE__, __LINE__);                                                  \
+    } while (0)
+
+constexpr int kWarps = 4;            // consumer warps of the attention kernel
+constexpr int kStages128 = 6;        // ring depth for head_dim 128 (6 x 32 KB)
+constexpr int kStages64 = 8;         // ring depth for head_dim 64  (8 x 16 KB)
+constexpr int kMaxProfile = 4096;
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool config_ok(const ckv_config *c, const char **why)
+{
+    *why = "";
+    if (!c) { *why = "config is NULL"; return false; }
+    if (c->num_layers < 1) { *why = "num_layers < 1"; return false; }
+    if (c->head_dim != 64 && c->head_dim != 128) { *why = "head_dim must be 64 or 128"; return false; }
+    if (c->page_size != ckv::kPageSize) { *why = "page_size must be 16"; return false; }
+    if (c->num_kv_heads < 1 || c->num_q_heads < 1 || c->num_q_heads % c->num_kv_heads != 0) {
+        *why = "num_q_heads must be a positive multiple of num_kv_heads"; return false;
+    }
+    if (c->num_q_heads / c->num_kv_heads > ckv::kMaxGroup) { *why = "group size above 8"; return false; }
+    if (c->num_pages < 1) { *why = "num_pages < 1"; return false; }
+    if (c->max_pages_per_req < 1) { *why = "max_pages_per_req < 1"; return false; }
+    if (c->max_batch < 1 || c->max_batch > ckv::kMaxBatch) { *why = "max_batch outside [1, 8192]"; return false; }
+    // TMA row coordinates are int32
+    const long long rows = (long long)c->num_layers * c->num_pages * c->num_kv_heads * 32;
+    if (rows >= (1ll << 31)) { *why = "pool has 2^31 or more rows"; return false; }
+    // tile counts are int32
+    const long long tiles = (long long)c->max_batch * c->num_kv_heads *
+                            (((long long)c->max_pages_per_req * ckv::kPageSize + ckv::kTileTokens - 1) / ckv::kTileTokens);
+    if (tiles >= (1ll << 31)) { *why = "max_batch * max context has 2^31 or more tiles"; return false; }
+    return true;
+}
+
+struct WorkspaceLayout {
+    size_t status, header, cta_start, tile_prefix, part_acc, part_ml;
+    size_t st_tables, st_lens, st_q, st_k, st_v, st_out;
+    size_t total;
+};
+
+WorkspaceLayout carve(const ckv_config &c)
+{
+    WorkspaceLayout w{};
+    size_t at = 0;
+    auto take = [&](size_t bytes) { size_t o = at; at = align_up(at + bytes, 256); return o; };
+    const size_t d2 = (size_t)c.head_dim * 2;
+    w.status = take(256);
+    w.header = take(sizeof(ckv::PlanHeader));
+    w.cta_start = take(sizeof(int4) * ckv::kMaxCtas);
+    w.tile_prefix = take(sizeof(int32_t) * ((size_t)c.max_batch + 1));
+    w.part_acc = take(sizeof(float) * 2 * ckv::kMaxCtas * ckv::kMaxGroup * c.head_dim);
+    w.part_ml = take(sizeof(float) * 2 * ckv::kMaxCtas * 2 * ckv::kMaxGroup);
+    w.st_tables = take(sizeof(int32_t) * (size_t)c.max_batch * c.max_pages_per_req);
+    w.st_lens = take(sizeof(int32_t) * (size_t)c.max_batch);
+    w.st_q = take((size_t)c.max_batch * c.num_q_heads * d2);
+    w.st_k = take((size_t)c.max_batch * c.num_kv_heads * d2);
+    w.st_v = take((size_t)c.max_batch * c.num_kv_heads * d2);
+    w.st_out = take((size_t)c.max_batch * c.num_q_heads * d2);
+    w.total = at;
+    return w;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct ckv_pool {
+    ckv_config cfg;
+    int device;
+    int num_sms;
+    int num_ctas;                    // partition width
+    uint8_t *d_pool;
+    uint8_t *d_ws;
+    WorkspaceLayout ws;
+    CUtensorMap tmap;
+    int64_t launches;
+    bool profile;
+    std::vector<cudaEvent_t> ev;     // pairs (start, stop)
+    int ev_used;
+
+    template <typename T> T *wsp(size_t off) const { return reinterpret_cast<T *>(d_ws + off); }
+};
+
+namespace {
+
+template <int D, int W, int S>
+int32_t launch_attention(ckv_pool *pool, const ckv::AttnParams &ap, cudaStream_t stream)
+{
+    using Lay = ckv::AttnLayout<D, W, S>;
+    static thread_local int configured_device = -1;
+    auto kernel = ckv::paged_decode_attn_kernel<D, W, S>;
+    if (configured_device != pool->device) {
+        CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
+        configured_device = pool->device;
+    }
+    kernel<<<pool->num_ctas, Lay::kThreads, Lay::kSmemBytes, stream>>>(pool->tmap, ap);
+    CKV_CUDA(cudaGetLastError());
+    return CKV_OK;
+}
+
+int32_t check_call(ckv_pool *pool, int32_t layer, int32_t batch, const char *fn)
+{
+    if (!pool) return fail(CKV_EINVAL, "%s: pool is NULL", fn);
+    if (layer < 0 || layer >= pool->cfg.num_layers)
+        return fail(CKV_EINVAL, "%s: layer %d outside [0, %d)", fn, layer, pool->cfg.num_layers);
+    if (batch < 1 || batch > pool->cfg.max_batch)
+        return fail(CKV_EINVAL, "%s: batch %d outside [1, %d]", fn, batch, pool->cfg.max_batch);
+    return CKV_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int32_t launch_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *d_out, cudaStream_t stream)
+{
+    const ckv_config &c = pool->cfg;
+    ckv::PlanParams pp{};
+    pp.seq_lens = d_seq_lens;
+    pp.header = pool->wsp<ckv::PlanHeader>(pool->ws.header);
+    pp.cta_start = pool->wsp<int4>(pool->ws.cta_start);
+    pp.tile_prefix = pool->wsp<int32_t>(pool->ws.tile_prefix);
+    pp.status = pool->wsp<uint32_t>(pool->ws.status);
+    pp.out = static_cast<uint16_t *>(d_out);
+    pp.batch = batch;
+    pp.max_pages_per_req = c.max_pages_per_req;
+    pp.num_kv_heads = c.num_kv_heads;
+    pp.num_ctas = pool->num_ctas;
+    pp.out_row_elems = c.num_q_heads * c.head_dim;
+    ckv::splitkv_plan_kernel<<<1, ckv::kPlanThreads, sizeof(int32_t) * ((size_t)batch + 1), stream>>>(pp);
+    CKV_CUDA(cudaGetLastError());
+    pool->launches += 1;
+    return CKV_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *ckv_last_error(void) { return g_error; }
+
+size_t kv_pool_bytes(const ckv_config *cfg)
+{
+    const char *why;
+    if (!config_ok(cfg, &why)) { fail(CKV_EINVAL, "kv_pool_bytes: %s", why); return 0; }
+    return (size_t)cfg->num_layers * cfg->num_pages * cfg->num_kv_heads * 2 * cfg->page_size * cfg->head_dim * 2;
+}
+
+size_t kv_workspace_bytes(const ckv_config *cfg)
+{
+    const char *why;
+    if (!config_ok(cfg, &why)) { fail(CKV_EINVAL, "kv_workspace_bytes: %s", why); return 0; }
+    return carve(*cfg).total;
+}
+
+int32_t kv_pool_create(const ckv_config *cfg, void *d_pool, size_t pool_bytes, void *d_workspace,
+                       size_t workspace_bytes, int32_t device, ckv_pool **out_pool)
+{
+    const char *why;
+    if (!out_pool) return fail(CKV_EINVAL, "kv_pool_create: out_pool is NULL");
+    *out_pool = nullptr;
+    if (!config_ok(cfg, &why)) return fail(CKV_EINVAL, "kv_pool_create: %s", why);
+    if (!d_pool || !d_workspace) return fail(CKV_EINVAL, "kv_pool_create: NULL device buffer");
+    if (reinterpret_cast<uintptr_t>(d_pool) & 255u) return fail(CKV_EINVAL, "kv_pool_create: d_pool not 256-byte aligned");
+    if (reinterpret_cast<uintptr_t>(d_workspace) & 255u) return fail(CKV_EINVAL, "kv_pool_create: d_workspace not 256-byte aligned");
+    if (pool_bytes < kv_pool_bytes(cfg)) return fail(CKV_ENOMEM, "kv_pool_create: pool buffer holds %zu bytes, %zu needed", pool_bytes, kv_pool_bytes(cfg));
+    const WorkspaceLayout ws = carve(*cfg);
+    if (workspace_bytes < ws.total) return fail(CKV_ENOMEM, "kv_pool_create: workspace holds %zu bytes, %zu needed", workspace_bytes, ws.total);
+    if (device < 0) return fail(CKV_EINVAL, "kv_pool_create: device < 0");
+
+    CKV_CUDA(cudaSetDevice(device));
+    int cc_major = 0, sms = 0;
+    CKV_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, device));
+    CKV_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    if (cc_major != 10) return fail(CKV_ECUDA, "kv_pool_create: device %d is sm_%dx; this library is built for sm_100a only", device, cc_major);
+
+    ckv_pool *p = new (std::nothrow) ckv_pool();
+    if (!p) return fail(CKV_ENOMEM, "kv_pool_create: host allocation failed");
+    p->cfg = *cfg;
+    p->device = device;
+    p->num_sms = sms;
+    p->num_ctas = std::min(sms, ckv::kMaxCtas);
+    p->d_pool = static_cast<uint8_t *>(d_pool);
+    p->d_ws = static_cast<uint8_t *>(d_workspace);
+    p->ws = ws;
+    p->launches = 0;
+    p->profile = false;
+    p->ev_used = 0;
+
+    // Tensor map over the whole pool seen as rows of head_dim bf16; one box = 32 rows (the 16 key
+    // rows and 16 value rows of one (page, kv head)) x 64 columns, stored with the 128-byte swizzle.
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+        delete p;
+        return fail(CKV_ECUDA, "kv_pool_create: cuTensorMapEncodeTiled not available (%s)", cudaGetErrorString(e));
+    }
+    const cuuint64_t rows = (cuuint64_t)cfg->num_layers * cfg->num_pages * cfg->num_kv_heads * 32;
+    const cuuint64_t dims[2] = {(cuuint64_t)cfg->head_dim, rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cfg->head_dim * 2};
+    const cuuint32_t box[2] = {64, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult cr = reinterpret_cast<EncodeTiledFn>(fn)(&p->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_pool, dims,
+                                                      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) {
+        delete p;
+        return fail(CKV_ECUDA, "kv_pool_create: cuTensorMapEncodeTiled returned %d", (int)cr);
+    }
+    cudaError_t me = cudaMemset(d_workspace, 0, ws.total);
+    if (me == cudaSuccess) me = cudaDeviceSynchronize();
+    if (me != cudaSuccess) {
+        delete p;
+        return fail(CKV_ECUDA, "kv_pool_create: clearing the workspace failed: %s", cudaGetErrorString(me));
+    }
+    *out_pool = p;
+    return CKV_OK;
+}
+
+int32_t kv_pool_destroy(ckv_pool *pool)
+{
+    if (!pool) return fail(CKV_EINVAL, "kv_pool_destroy: pool is NULL");
+    cudaSetDevice(pool->device);
+    cudaDeviceSynchronize();
+    for (cudaEvent_t ev : pool->ev) cudaEventDestroy(ev);
+    delete pool;
+    return CKV_OK;
+}
+
+int32_t ckv_set_partition(ckv_pool *pool, int32_t num_ctas)
+{
+    if (!pool) return fail(CKV_EINVAL, "ckv_set_partition: pool is NULL");
+    if (num_ctas < 1 || num_ctas > ckv::kMaxCtas) return fail(CKV_EINVAL, "ckv_set_partition: %d outside [1, %d]", num_ctas, ckv::kMaxCtas);
+    pool->num_ctas = num_ctas;
+    return CKV_OK;
+}
+
+int32_t ckv_get_partition(const ckv_pool *pool) { return pool ? pool->num_ctas : CKV_EINVAL; }
+
+int64_t ckv_launch_count(const ckv_pool *pool) { return pool ? pool->launches : 0; }
+
+int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
+                  const int32_t *d_seq_lens, const void *d_k_new, const void *d_v_new, void *stream)
+{
+    if (int32_t rc = check_call(pool, layer, batch, "kv_append")) return rc;
+    if (!d_block_tables || !d_seq_lens || !d_k_new || !d_v_new) return fail(CKV_EINVAL, "kv_append: NULL argument");
+    if (!aligned16(d_k_new) || !aligned16(d_v_new)) return fail(CKV_EINVAL, "kv_append: k_new/v_new not 16-byte aligned");
+    const ckv_config &c = pool->cfg;
+    ckv::AppendParams ap{};
+    const size_t layer_bytes = (size_t)c.num_pages * c.num_kv_heads * 2 * c.page_size * c.head_dim * 2;
+    ap.pool_layer = reinterpret_cast<uint4 *>(pool->d_pool + layer_bytes * layer);
+    ap.block_tables = d_block_tables;
+    ap.seq_lens = d_seq_lens;
+    ap.k_new = static_cast<const uint4 *>(d_k_new);
+    ap.v_new = static_cast<const uint4 *>(d_v_new);
+    ap.status = pool->wsp<uint32_t>(pool->ws.status);
+    ap.batch = batch;
+    ap.max_pages_per_req = c.max_pages_per_req;
+    ap.num_pages = c.num_pages;
+    ap.num_kv_heads = c.num_kv_heads;
+    ap.head_dim = c.head_dim;
+    const long long work = (long long)batch * c.num_kv_heads * 2 * (c.head_dim / 8);
+    const int threads = 256;
+    const int blocks = (int)std::min<long long>((work + threads - 1) / threads, 4096);
+    ckv::kv_append_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(stream)>>>(ap);
+    CKV_CUDA(cudaGetLastError());
+    pool->launches += 1;
+    return CKV_OK;
+}
+
+int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
+                         const int32_t *d_seq_lens, const void *d_q, void *d_out, void *stream)
+{
+    if (int32_t rc = check_call(pool, layer, batch, "decode_attention")) return rc;
+    if (!d_block_tables || !d_seq_lens || !d_q || !d_out) return fail(CKV_EINVAL, "decode_attention: NULL argument");
+    if (!aligned16(d_q) || !aligned16(d_out)) return fail(CKV_EINVAL, "decode_attention: q/out not 16-byte aligned");
+    const ckv_config &c = pool->cfg;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    if (int32_t rc = launch_plan(pool, batch, d_seq_lens, d_out, s)) return rc;
+
+    ckv::AttnParams ap{};
+    ap.block_tables = d_block_tables;
+    ap.seq_lens = d_seq_lens;
+    ap.q = static_cast<const uint16_t *>(d_q);
+    ap.out = static_cast<uint16_t *>(d_out);
+    ap.header = pool->wsp<ckv::PlanHeader>(pool->ws.header);
+    ap.cta_start = pool->wsp<int4>(pool->ws.cta_start);
+    ap.part_acc = pool->wsp<float>(pool->ws.part_acc);
+    ap.part_ml = pool->wsp<float>(pool->ws.part_ml);
+    ap.status = pool->wsp<uint32_t>(pool->ws.status);
+    ap.batch = batch;
+    ap.max_pages_per_req = c.max_pages_per_req;
+    ap.num_pages = c.num_pages;
+    ap.num_kv_heads = c.num_kv_heads;
+    ap.num_q_heads = c.num_q_heads;
+    ap.group = c.num_q_heads / c.num_kv_heads;
+    ap.layer_page_base = layer * c.num_pages;
+    ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
+
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if (pool->profile && pool->ev_used < kMaxProfile) {
+        if ((size_t)(2 * pool->ev_used + 2) > pool->ev.size()) {
+            cudaEvent_t a, b;
+            CKV_CUDA(cudaEventCreate(&a));
+            CKV_CUDA(cudaEventCreate(&b));
+            pool->ev.push_back(a);
+            pool->ev.push_back(b);
+        }
+        ev0 = pool->ev[2 * pool->ev_used];
+        ev1 = pool->ev[2 * pool->ev_used + 1];
+        pool->ev_used += 1;
+        CKV_CUDA(cudaEventRecord(ev0, s));
+    }
+    int32_t rc;
+    if (c.head_dim == 128) rc = launch_attention<128, kWarps, kStages128>(pool, ap, s);
+    else rc = launch_attention<64, kWarps, kStages64>(pool, ap, s);
+    if (rc) return rc;
+    if (ev1) CKV_CUDA(cudaEventRecord(ev1, s));
+    pool->launches += 1;
+
+    if (pool->num_ctas > 1) {
+        ckv::CombineParams cp{};
+        cp.header = ap.header;
+        cp.tile_prefix = pool->wsp<int32_t>(pool->ws.tile_prefix);
+        cp.part_acc = ap.part_acc;
+        cp.part_ml = ap.part_ml;
+        cp.out = ap.out;
+        cp.batch = batch;
+        cp.num_kv_heads = c.num_kv_heads;
+        cp.num_q_heads = c.num_q_heads;
+        cp.group = ap.group;
+        cp.head_dim = c.head_dim;
+        ckv::lse_combine_kernel<<<pool->num_ctas - 1, 256, 0, s>>>(cp);
+        CKV_CUDA(cudaGetLastError());
+        pool->launches += 1;
+    }
+    return CKV_OK;
+}
+
+int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *stream,
+                    int32_t *h_header, int32_t *h_cta_start)
+{
+    if (int32_t rc = check_call(pool, 0, batch, "decode_plan")) return rc;
+    if (!d_seq_lens || !h_header || !h_cta_start) return fail(CKV_EINVAL, "decode_plan: NULL argument");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (int32_t rc = launch_plan(pool, batch, d_seq_lens, nullptr, s)) return rc;
+    CKV_CUDA(cudaMemcpyAsync(h_header, pool->d_ws + pool->ws.header, sizeof(ckv::PlanHeader), cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaMemcpyAsync(h_cta_start, pool->d_ws + pool->ws.cta_start, sizeof(int4) * pool->num_ctas, cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaStreamSynchronize(s));
+    return CKV_OK;
+}
+
+int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits)
+{
+    if (!pool) return fail(CKV_EINVAL, "kv_check_status: pool is NULL");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    uint32_t bits = 0;
+    CKV_CUDA(cudaMemcpyAsync(&bits, pool->d_ws + pool->ws.status, sizeof bits, cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaMemsetAsync(pool->d_ws + pool->ws.status, 0, sizeof bits, s));
+    CKV_CUDA(cudaStreamSynchronize(s));
+    if (out_bits) *out_bits = bits;
+    if (bits & ckv::kStatusWaitLimit) return fail(CKV_ETIMEOUT, "device status 0x%x: a bounded wait gave up", bits);
+    if (bits & (ckv::kStatusBadLength | ckv::kStatusBadPage))
+        return fail(CKV_EBOUNDS, "device status 0x%x: %s%s", bits, (bits & ckv::kStatusBadLength) ? "[context length out of range]" : "",
+                    (bits & ckv::kStatusBadPage) ? "[page id out of range]" : "");
+    return CKV_OK;
+}
+
+int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *h_block_tables,
+                         const int32_t *h_seq_lens, const void *h_q, const void *h_k_new,
+                         const void *h_v_new, void *h_out, void *stream)
+{
+    if (int32_t rc = check_call(pool, layer, batch, "decode_step_host")) return rc;
+    if (!h_block_tables || !h_seq_lens || !h_q || !h_k_new || !h_v_new || !h_out)
+        return fail(CKV_EINVAL, "decode_step_host: NULL argument");
+    const ckv_config &c = pool->cfg;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t d2 = (size_t)c.head_dim * 2;
+    int32_t *d_bt = pool->wsp<int32_t>(pool->ws.st_tables);
+    int32_t *d_sl = pool->wsp<int32_t>(pool->ws.st_lens);
+    void *d_q = pool->d_ws + pool->ws.st_q, *d_k = pool->d_ws + pool->ws.st_k;
+    void *d_v = pool->d_ws + pool->ws.st_v, *d_o = pool->d_ws + pool->ws.st_out;
+    CKV_CUDA(cudaMemcpyAsync(d_bt, h_block_tables, sizeof(int32_t) * (size_t)batch * c.max_pages_per_req, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(d_sl, h_seq_lens, sizeof(int32_t) * (size_t)batch, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(d_q, h_q, (size_t)batch * c.num_q_heads * d2, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(d_k, h_k_new, (size_t)batch * c.num_kv_heads * d2, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(d_v, h_v_new, (size_t)batch * c.num_kv_heads * d2, cudaMemcpyHostToDevice, s));
+    if (int32_t rc = kv_append(pool, layer, batch, d_bt, d_sl, d_k, d_v, stream)) return rc;
+    if (int32_t rc = decode_attention(pool, layer, batch, d_bt, d_sl, d_q, d_o, stream)) return rc;
+    CKV_CUDA(cudaMemcpyAsync(h_out, d_o, (size_t)batch * c.num_q_heads * d2, cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaStreamSynchronize(s));
+    return CKV_OK;
+}
+
+int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch_sizes, int32_t batch_stride,
+                           const int32_t *d_block_tables, const int32_t *d_seq_lens, const void *d_q,
+                           const void *d_k_new, const void *d_v_new, void *d_out, int32_t warmup,
+                           int32_t iters, void *d_flush, size_t flush_bytes, void *stream,
+                           double *out_median_us, double *out_min_us)
+{
+    if (!pool) return fail(CKV_EINVAL, "step_latency_sweep: pool is NULL");
+    if (n_sizes < 1 || !batch_sizes || !out_median_us || !out_min_us) return fail(CKV_EINVAL, "step_latency_sweep: bad size list or outputs");
+    if (warmup < 0 || iters < 1 || iters > 100000) return fail(CKV_EINVAL, "step_latency_sweep: bad warmup/iters");
+    if (batch_stride < 1 || batch_stride > pool->cfg.max_batch) return fail(CKV_EINVAL, "step_latency_sweep: bad batch_stride");
+    for (int i = 0; i < n_sizes; ++i)
+        if (batch_sizes[i] < 1 || batch_sizes[i] > batch_stride) return fail(CKV_EINVAL, "step_latency_sweep: batch size %d outside [1, %d]", batch_sizes[i], batch_stride);
+    if (!d_block_tables || !d_seq_lens || !d_q || !d_k_new || !d_v_new || !d_out) return fail(CKV_EINVAL, "step_latency_sweep: NULL argument");
+    const ckv_config &c = pool->cfg;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t d2 = (size_t)c.head_dim * 2;
+    const size_t q_layer = (size_t)batch_stride * c.num_q_heads * d2;
+    const size_t kv_layer = (size_t)batch_stride * c.num_kv_heads * d2;
+
+    std::vector<cudaEvent_t> ev(2 * (size_t)iters);
+    for (auto &e : ev) CKV_CUDA(cudaEventCreate(&e));
+    int32_t rc = CKV_OK;
+    std::vector<float> ms((size_t)iters);
+    for (int i = 0; i < n_sizes && rc == CKV_OK; ++i) {
+        const int32_t b = batch_sizes[i];
+        for (int k = 0; k < warmup + iters && rc == CKV_OK; ++k) {
+            const bool timed = k >= warmup;
+            if (d_flush && flush_bytes) {
+                cudaError_t e = cudaMemsetAsync(d_flush, k & 0xff, flush_bytes, s);
+                if (e != cudaSuccess) { rc = fail(CKV_ECUDA, "flush memset failed: %s", cudaGetErrorString(e)); break; }
+            }
+            if (timed) cudaEventRecord(ev[2 * (size_t)(k - warmup)], s);
+            for (int layer = 0; layer < c.num_layers && rc == CKV_OK; ++layer) {
+                const uint8_t *q = static_cast<const uint8_t *>(d_q) + q_layer * layer;
+                const uint8_t *kn = static_cast<const uint8_t *>(d_k_new) + kv_layer * layer;
+                const uint8_t *vn = static_cast<const uint8_t *>(d_v_new) + kv_layer * layer;
+                uint8_t *o = static_cast<uint8_t *>(d_out) + q_layer * layer;
+                rc = kv_append(pool, layer, b, d_block_tables, d_seq_lens, kn, vn, stream);
+                if (rc == CKV_OK) rc = decode_attention(pool, layer, b, d_block_tables, d_seq_lens, q, o, stream);
+            }
+            if (timed) cudaEventRecord(ev[2 * (size_t)(k - warmup) + 1], s);
+        }
+        if (rc != CKV_OK) break;
+        cudaError_t e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) { rc = fail(CKV_ECUDA, "step_latency_sweep: synchronise failed: %s", cudaGetErrorString(e)); break; }
+        for (int k = 0; k < iters; ++k) cudaEventElapsedTime(&ms[k], ev[2 * (size_t)k], ev[2 * (size_t)k + 1]);
+        std::vector<float> sorted(ms);
+        std::sort(sorted.begin(), sorted.end());
+        const double med = (iters & 1) ? sorted[iters / 2] : 0.5 * (sorted[iters / 2 - 1] + sorted[iters / 2]);
+        out_median_us[i] = med * 1000.0;
+        out_min_us[i] = sorted[0] * 1000.0;
+    }
+    for (auto &e : ev) cudaEventDestroy(e);
+    if (rc != CKV_OK) return rc;
+    return kv_check_status(pool, stream, nullptr);
+}
+
+int32_t ckv_profile_enable(ckv_pool *pool, int32_t enable)
+{
+    if (!pool) return fail(CKV_EINVAL, "ckv_profile_enable: pool is NULL");
+    pool->profile = enable != 0;
+    pool->ev_used = 0;
+    return CKV_OK;
+}
+
+int32_t ckv_profile_read(ckv_pool *pool, double *out_attention_ms, int32_t *out_launches)
+{
+    if (!pool || !out_attention_ms || !out_launches) return fail(CKV_EINVAL, "ckv_profile_read: NULL argument");
+    CKV_CUDA(cudaSetDevice(pool->device));
+    CKV_CUDA(cudaDeviceSynchronize());
+    double total = 0.0;
+    for (int i = 0; i < pool->ev_used; ++i) {
+        float ms = 0.f;
+        CKV_CUDA(cudaEventElapsedTime(&ms, pool->ev[2 * i], pool->ev[2 * i + 1]));
+        total += ms;
+    }
+    *out_attention_ms = total;
+    *out_launches = pool->ev_used;
+    return CKV_OK;
+}
+
+}  // extern "C"

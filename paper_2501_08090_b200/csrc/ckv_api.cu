@@ -34,9 +34,9 @@ int32_t fail(int32_t code, const char *fmt, ...)
                         __FILE__, __LINE__);                                                  \
     } while (0)
 
-constexpr int kWarps = 4;            // consumer warps of the attention kernel
-constexpr int kStages128 = 6;        // ring depth for head_dim 128 (6 x 32 KB)
-constexpr int kStages64 = 8;         // ring depth for head_dim 64  (8 x 16 KB)
+// Attention kernel shapes: ring depth is a multiple of the consumer-warp count (see the kernel).
+constexpr int kWarps128 = 6, kStages128 = 6;     // head_dim 128: 6 x 32 KB in flight per SM
+constexpr int kWarps64 = 4, kStages64 = 8;       // head_dim 64:  8 x 16 KB
 constexpr int kMaxProfile = 4096;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -349,8 +349,8 @@ int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int
         CKV_CUDA(cudaEventRecord(ev0, s));
     }
     int32_t rc;
-    if (c.head_dim == 128) rc = launch_attention<128, kWarps, kStages128>(pool, ap, s);
-    else rc = launch_attention<64, kWarps, kStages64>(pool, ap, s);
+    if (c.head_dim == 128) rc = launch_attention<128, kWarps128, kStages128>(pool, ap, s);
+    else rc = launch_attention<64, kWarps64, kStages64>(pool, ap, s);
     if (rc) return rc;
     if (ev1) CKV_CUDA(cudaEventRecord(ev1, s));
     pool->launches += 1;

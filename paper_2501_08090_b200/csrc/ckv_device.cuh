@@ -377,6 +377,11 @@ __global__ void __launch_bounds__((W + 1) * 32, 1)
 paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnParams p)
 {
     using Lay = AttnLayout<D, W, S>;
+    // Stage `it` lives in slot it % S and is consumed by warp it % W.  A consumer tells "my data
+    // has landed" from the parity of the slot's barrier, which is only unambiguous if it cannot
+    // get a whole phase ahead of the slot's previous use.  Copies complete out of order, so that
+    // holds only when the previous use of the slot was consumed by the SAME warp: S % W == 0.
+    static_assert(S % W == 0, "every ring slot must always be consumed by the same warp");
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     float *scratch_o = (float *)(smem + S * Lay::kStageBytes);            // [W][D][8]

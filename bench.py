@@ -1,0 +1,424 @@
+#!/usr/bin/env python
+"""Benchmark of the decode-iteration hot path: KV append + paged GQA decode attention.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-sweep]
+
+One step = one pass of the whole hot path (append, split-KV plan, partial attention, combine) for
+every layer of the workload over one seeded synthetic batch.  The headline workload is the
+Llama-3-8B-shaped layer at batch 64 with contexts uniform in [512, 4096] ("llama8b_b64",
+~600 MB of KV per step, several times the L2 size, so every step streams from HBM).
+
+Prints ONE JSON line (rank 0).  `value` is the algorithmic bytes all ranks moved per second of
+the slowest rank's device time, in TB/s; with N > 1 every rank is an independent serving
+instance with its own batch (weak scaling, no collective on the data path).
+
+`--impl reference` times the fp64 CPU oracle on the host cores instead, on a bounded sample of
+the same workload (a deliberately slow baseline, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2501_08090_b200 import workloads as wl  # noqa: E402
+
+HEADLINE = "llama8b_b64"
+METRIC = "decode_attention_hbm_bandwidth"
+UNIT = "TB/s"
+NORMALISED_TO_TBS = 8.0          # the metric is quoted as a fraction of 8 TB/s
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ------------------------------------------------------------------------------- clocks
+
+class ClockSampler(threading.Thread):
+    """Polls SM clock and clock-event reasons through NVML while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown",
+               0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, device_index: int, period_s: float = 0.002):
+        super().__init__(daemon=True)
+        self.period = period_s
+        self.samples, self.reason_bits = [], 0
+        self.max_mhz = None
+        self.error = None
+        self._stop_evt = threading.Event()
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            except Exception:
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(device_index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # pragma: no cover - depends on the box
+            self.error = repr(e)
+
+    def _poll(self):
+        nv = self.nv
+        self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+        try:
+            self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h))
+        except Exception:
+            self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+
+    def run(self):
+        if self._h is None:
+            return
+        while not self._stop_evt.is_set():
+            try:
+                self._poll()
+            except Exception as e:  # pragma: no cover
+                self.error = repr(e)
+                return
+            time.sleep(self.period)
+
+    def stop(self) -> dict:
+        self._stop_evt.set()
+        self.join(timeout=2.0)
+        reasons = [name for bit, name in self.REASONS.items() if self.reason_bits & bit]
+        out = {"sm_mhz": int(statistics.median(self.samples)) if self.samples else None,
+               "sm_max_mhz": self.max_mhz, "reasons": reasons, "samples": len(self.samples)}
+        if self.error:
+            out["error"] = self.error
+        return out
+
+
+# ------------------------------------------------------------------------------- device workload
+
+class DeviceWorkload:
+    """A workload drawn on the GPU: pool, tables, per-layer q / k_new / v_new / out."""
+
+    def __init__(self, name: str, device, seed_offset: int = 0, batch=None, num_layers=None):
+        import torch
+        from paper_2501_08090_b200 import binding
+        w = wl.workload(name) if num_layers is None else wl.workload(name, num_layers=num_layers)
+        if seed_offset:
+            w = wl.workload(name, seed=w.seed + 1000 * seed_offset,
+                            **({"num_layers": num_layers} if num_layers is not None else {}))
+        self.w, self.device = w, device
+        self.lens = wl.seq_lens(w, batch)
+        self.B = int(self.lens.size)
+        self.num_pages = wl.num_pool_pages(w, self.lens)
+        self.bt_host = wl.block_tables(self.lens, self.num_pages, w.seed, w.page_size)
+        cfg = binding.make_config(w.num_layers, w.num_q_heads, w.num_kv_heads, w.head_dim,
+                                  self.num_pages, self.bt_host.shape[1], self.B)
+        pool = wl.device_normal_bf16((wl.pool_elems(w, self.num_pages),), w.seed, 1, device)
+        self.kp = binding.KvPool(cfg, device=device, pool=pool)
+        self.bt = torch.from_numpy(self.bt_host).to(device)
+        self.sl = torch.from_numpy(self.lens).to(device)
+        self.q = wl.device_normal_bf16((w.num_layers, self.B, w.num_q_heads, w.head_dim), w.seed, 2, device)
+        self.k_new = wl.device_normal_bf16((w.num_layers, self.B, w.num_kv_heads, w.head_dim), w.seed, 3, device)
+        self.v_new = wl.device_normal_bf16((w.num_layers, self.B, w.num_kv_heads, w.head_dim), w.seed, 4, device)
+        self.out = torch.zeros_like(self.q)
+        self.bytes = wl.algorithmic_bytes(w, self.lens)
+
+    def step_calls(self):
+        """Pre-marshalled (function, args) pairs of one step, so the timed loop is two C calls per layer."""
+        import torch
+        from paper_2501_08090_b200 import binding
+        lib, h = binding.lib, self.kp._h
+        s = torch.cuda.current_stream().cuda_stream
+        calls = []
+        for layer in range(self.w.num_layers):
+            calls.append((lib.kv_append, (h, layer, self.B, self.bt.data_ptr(), self.sl.data_ptr(),
+                                          self.k_new[layer].data_ptr(), self.v_new[layer].data_ptr(), s)))
+            calls.append((lib.decode_attention, (h, layer, self.B, self.bt.data_ptr(), self.sl.data_ptr(),
+                                                 self.q[layer].data_ptr(), self.out[layer].data_ptr(), s)))
+        return calls
+
+    def run_steps(self, n: int) -> None:
+        from paper_2501_08090_b200 import binding
+        calls = self.step_calls()
+        for _ in range(n):
+            for fn, args in calls:
+                rc = fn(*args)
+                if rc != 0:
+                    raise binding.CkvError(rc, binding.last_error())
+
+
+def dist_setup(n_gpus: int):
+    """(rank, world, local_rank); initialises NCCL only when launched under torchrun."""
+    import torch
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group(backend="nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    return rank, world, local
+
+
+def reduce_max_sum(t_ms: float, units: float, world: int):
+    """Max over ranks of the time, sum over ranks of the units (bytes, launches ...)."""
+    if world == 1:
+        return t_ms, units
+    import torch
+    import torch.distributed as dist
+    a = torch.tensor([t_ms], dtype=torch.float64, device="cuda")
+    b = torch.tensor([units], dtype=torch.float64, device="cuda")
+    dist.all_reduce(a, op=dist.ReduceOp.MAX)
+    dist.all_reduce(b, op=dist.ReduceOp.SUM)
+    return float(a.item()), float(b.item())
+
+
+def barrier(world: int):
+    import torch
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+def timed_region(fn, world: int, device_index: int):
+    """barrier+sync, CUDA events on the launch stream around fn(), barrier+sync; returns (ms, clocks)."""
+    import torch
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier(world)
+    sampler = ClockSampler(device_index)
+    sampler.start()
+    ev0.record()
+    fn()
+    ev1.record()
+    barrier(world)
+    clocks = sampler.stop()
+    return ev0.elapsed_time(ev1), clocks
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------------------- CPU baseline (oracle)
+
+def oracle_sample_inputs(name: str, rows):
+    """Host inputs for the chosen requests of a workload, as a compact pool (oracle's arm only)."""
+    w = wl.workload(name)
+    lens_all = wl.seq_lens(w)
+    lens = lens_all[list(rows)]
+    npg = int(wl.pages_of(lens).sum())
+    bt = wl.block_tables(lens, npg, w.seed)
+    b = lens.size
+    return dict(w=w, lens=lens, num_pages=npg, bt=bt,
+                pool=wl.normal_bf16((wl.pool_elems(w, npg, 1),), w.seed, 11),
+                q=wl.normal_bf16((b, w.num_q_heads, w.head_dim), w.seed, 12),
+                k=wl.normal_bf16((b, w.num_kv_heads, w.head_dim), w.seed, 13),
+                v=wl.normal_bf16((b, w.num_kv_heads, w.head_dim), w.seed, 14))
+
+
+def oracle_step(inp) -> float:
+    """One oracle pass (append + attention) over the sample; seconds."""
+    from oracle import oracle
+    from oracle.oracle import PoolShape
+    w = inp["w"]
+    sh = PoolShape(1, inp["num_pages"], w.num_q_heads, w.num_kv_heads, w.page_size, w.head_dim)
+    t0 = time.perf_counter()
+    rc = oracle.kv_append(inp["pool"], sh, 0, inp["bt"], inp["lens"], inp["k"], inp["v"])
+    assert rc == 0
+    oracle.decode_attention(inp["pool"], sh, 0, inp["bt"], inp["lens"], inp["q"])
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(name: str, target_s: float = 12.0) -> dict:
+    """The oracle as it stands, timed on the host cores on a bounded sample of the workload."""
+    from oracle import oracle
+    w = wl.workload(name)
+    total = w.batch
+    probe = oracle_sample_inputs(name, range(min(2, total)))
+    t_probe = oracle_step(probe)
+    n = int(max(1, min(total, round(len(probe["lens"]) * target_s / max(t_probe, 1e-6)))))
+    inp = oracle_sample_inputs(name, range(n))
+    oracle_step(inp)                                   # untimed first pass (page faults, thread start)
+    times = []
+    while len(times) < 3 or (sum(times) < target_s and len(times) < 50):
+        times.append(oracle_step(inp))
+    t = sum(times) / len(times)
+    nbytes = wl.algorithmic_bytes(w, inp["lens"], 1)["total"]
+    return {"value": nbytes / t / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "first %d of %d requests of %s, one layer; mean of %d passes (%.1f s of CPU work)"
+                      % (n, total, name, len(times), sum(times)),
+            "us_per_step_sample": t * 1e6}
+
+
+def run_reference(args) -> None:
+    """--impl reference: K timed oracle steps on a sample sized so the run ends within minutes."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle
+    w = wl.workload(HEADLINE)
+    budget_s = 150.0
+    one = oracle_sample_inputs(HEADLINE, range(1))
+    t_one = min(oracle_step(one), oracle_step(one))
+    per_step = budget_s / max(1, args.steps + args.warmup)
+    n = int(max(1, min(w.batch, per_step / max(t_one, 1e-6))))
+    inp = oracle_sample_inputs(HEADLINE, range(n))
+    for _ in range(args.warmup):
+        oracle_step(inp)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(inp)
+    dt = time.perf_counter() - t0
+    nbytes = wl.algorithmic_bytes(w, inp["lens"], 1)["total"]
+    value = nbytes * args.steps / dt / 1e12
+    sample = "first %d of %d requests of %s per step" % (n, w.batch, HEADLINE)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic",
+            "config": {"workload": HEADLINE, "sample": sample, "device": "host cpu"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------- our arm
+
+def run_ours(args) -> None:
+    import torch
+    from paper_2501_08090_b200 import binding   # raises if the CUDA library is missing
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (sm_100a); there is no CPU path")
+    rank, world, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local if world > 1 else 0)
+    dw = DeviceWorkload(HEADLINE, dev, seed_offset=rank)
+    w = dw.w
+    K, W = args.steps, max(args.warmup, 3)
+
+    # ---- headline: K steps back to back, inputs resident in HBM
+    dw.run_steps(W)
+    dw.kp.check_status()
+    n0 = dw.kp.launch_count()
+    ms, clocks = timed_region(lambda: dw.run_steps(K), world, dev.index or 0)
+    launches = dw.kp.launch_count() - n0
+    dw.kp.check_status()
+    ms_max, bytes_all = reduce_max_sum(ms, float(dw.bytes["total"]) * K, world)
+    _, launches_all = reduce_max_sum(0.0, float(launches), world)
+    _, tokens_all = reduce_max_sum(0.0, float(dw.B) * K, world)
+    _, kv_all = reduce_max_sum(0.0, float(dw.bytes["kv"]) * K, world)
+    value = bytes_all / (ms_max * 1e-3) / 1e12
+
+    # ---- dominant kernel alone: CUDA events around every attention launch (second pass)
+    P = min(K, 2000)
+    dw.kp.profile_enable(True)
+    dw.run_steps(P)
+    attn_ms, attn_n = dw.kp.profile_read()
+    dw.kp.profile_enable(False)
+    attn_bytes = (dw.bytes["kv"] + dw.bytes["q_out"] + dw.bytes["tables"]) // w.num_layers
+    peak, peak_kind = measured_peak_gbs()
+    achieved = attn_bytes / (attn_ms / attn_n * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "paged_decode_attn_kernel", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_kind": "of " + peak_kind,
+                "traffic": None, "bytes_per_launch": attn_bytes, "us_per_launch": attn_ms / attn_n * 1e3,
+                "frac_of_8TBs": achieved / (NORMALISED_TO_TBS * 1e3)}
+
+    # ---- end to end through the host-buffer entry point (pinned memory, copies inside the timing)
+    E = min(K, 500)
+    pin = lambda t: t.cpu().pin_memory()
+    hb = dict(bt=pin(dw.bt), sl=pin(dw.sl), q=pin(dw.q[0]), k=pin(dw.k_new[0]), v=pin(dw.v_new[0]))
+    hout = torch.zeros_like(hb["q"]).pin_memory()
+    h2d = sum(hb[k].numel() * hb[k].element_size() for k in hb)
+    d2h = hout.numel() * hout.element_size()
+
+    def e2e_steps(n):
+        for _ in range(n):
+            for layer in range(w.num_layers):
+                dw.kp.decode_step_host(layer, hb["bt"], hb["sl"], hb["q"], hb["k"], hb["v"], hout)
+    e2e_steps(3)
+    barrier(world)
+    t0 = time.perf_counter()
+    e2e_steps(E)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    e2e_ms_max, e2e_bytes = reduce_max_sum(e2e_s * 1e3, float(dw.bytes["total"]) * E, world)
+    e2e = {"value": e2e_bytes / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d * w.num_layers,
+           "d2h_bytes_per_step": d2h * w.num_layers, "steps": E, "us_per_step": e2e_ms_max / E * 1e3}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": ms_max / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": HEADLINE, "batch": dw.B, "layers": w.num_layers, "q_heads": w.num_q_heads,
+                   "kv_heads": w.num_kv_heads, "head_dim": w.head_dim, "page_size": w.page_size,
+                   "context": "uniform[512,4096]", "tokens_in_context": int(dw.lens.sum()),
+                   "l2": "inputs larger than L2 (%.0f MB of KV per step)" % (dw.bytes["kv"] / 1e6),
+                   "instances": "one independent batch per GPU"},
+        "us_per_step": ms_max / K * 1e3, "tokens_per_s": tokens_all / (ms_max * 1e-3),
+        "kv_gbs": kv_all / (ms_max * 1e-3) / 1e9, "frac_of_8TBs": value / NORMALISED_TO_TBS,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches_all), "roofline": roofline,
+    }
+
+    if rank == 0 and world == 1:
+        if not args.no_sweep:
+            line["latency_sweep"] = run_sweep(dev)
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(HEADLINE)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def run_sweep(dev) -> dict:
+    """Latency against batch size on the mixed interactive/batch workload (nested prefixes)."""
+    import torch
+    del_later = DeviceWorkload("mixed_sweep", dev)
+    dw = del_later
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # larger than the L2
+    sizes = list(wl.SWEEP_BATCH_SIZES)
+    med, mn = dw.kp.step_latency_sweep(sizes, dw.bt, dw.sl, dw.q, dw.k_new, dw.v_new, dw.out,
+                                       warmup=3, iters=20, flush=flush)
+    rows = []
+    for b, m, lo in zip(sizes, med.tolist(), mn.tolist()):
+        nb = wl.algorithmic_bytes(dw.w, dw.lens[:b])["total"]
+        rows.append({"batch": b, "us_per_step": round(m, 2), "us_min": round(lo, 2),
+                     "tokens_per_s": round(b / (m * 1e-6)), "tbs": round(nb / (m * 1e-6) / 1e12, 3)})
+    dw.kp.close()
+    return {"workload": "mixed_sweep", "l2": "256 MB flush before every timed step", "points": rows}
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the batch-size latency sweep")
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiling runs)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -179,6 +179,14 @@ int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch
 int32_t ckv_profile_enable(ckv_pool *pool, int32_t enable);
 int32_t ckv_profile_read(ckv_pool *pool, double *out_attention_ms, int32_t *out_launches);
 
+/*
+ * Per-CTA timeline of the most recent attention kernel, for load-balance analysis (synchronises
+ * `stream`).  h_trace: uint64 [ckv_get_partition()][4], nanoseconds of the GPU's global timer:
+ * CTA start, first tile consumed (0 if the CTA had no work), producer warp done, consumers done.
+ * Errors: CKV_EINVAL, CKV_ECUDA.
+ */
+int32_t ckv_read_cta_trace(ckv_pool *pool, void *stream, uint64_t *h_trace);
+
 /* Kernels launched through this handle since creation (append, plan, attention, combine). */
 int64_t ckv_launch_count(const ckv_pool *pool);
 

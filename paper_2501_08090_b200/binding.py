@@ -23,7 +23,7 @@ EXPORTS = (
     "kv_pool_bytes", "kv_workspace_bytes", "kv_pool_create", "kv_pool_destroy", "kv_append",
     "decode_attention", "decode_plan", "ckv_set_partition", "ckv_get_partition", "kv_check_status",
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
-    "ckv_launch_count", "ckv_last_error",
+    "ckv_launch_count", "ckv_last_error", "ckv_read_cta_trace",
 )
 
 
@@ -64,6 +64,7 @@ def _load() -> ctypes.CDLL:
     lib.ckv_profile_enable.restype = i32; lib.ckv_profile_enable.argtypes = [vp, i32]
     lib.ckv_profile_read.restype = i32
     lib.ckv_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
+    lib.ckv_read_cta_trace.restype = i32; lib.ckv_read_cta_trace.argtypes = [vp, vp, vp]
     lib.ckv_launch_count.restype = i64; lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_last_error.restype = ctypes.c_char_p; lib.ckv_last_error.argtypes = []
     return lib
@@ -224,6 +225,12 @@ class KvPool:
         n = ctypes.c_int32(0)
         _check(lib.ckv_profile_read(self._h, ctypes.byref(ms), ctypes.byref(n)))
         return float(ms.value), int(n.value)
+
+    def read_cta_trace(self, stream=None) -> np.ndarray:
+        """uint64 [num_ctas][4] ns: CTA start, first tile consumed, producer done, consumers done."""
+        trace = np.zeros((self.get_partition(), 4), dtype=np.uint64)
+        _check(lib.ckv_read_cta_trace(self._h, _stream_ptr(stream), trace.ctypes.data))
+        return trace
 
     def launch_count(self) -> int:
         return int(lib.ckv_launch_count(self._h))

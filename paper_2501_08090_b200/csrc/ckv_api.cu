@@ -66,7 +66,7 @@ bool config_ok(const ckv_config *c, const char **why)
 }
 
 struct WorkspaceLayout {
-    size_t status, header, cta_start, tile_prefix, part_acc, part_ml;
+    size_t status, header, cta_start, tile_prefix, part_acc, part_ml, cta_trace;
     size_t st_tables, st_lens, st_q, st_k, st_v, st_out;
     size_t total;
 };
@@ -83,6 +83,7 @@ WorkspaceLayout carve(const ckv_config &c)
     w.tile_prefix = take(sizeof(int32_t) * ((size_t)c.max_batch + 1));
     w.part_acc = take(sizeof(float) * 2 * ckv::kMaxCtas * ckv::kMaxGroup * c.head_dim);
     w.part_ml = take(sizeof(float) * 2 * ckv::kMaxCtas * 2 * ckv::kMaxGroup);
+    w.cta_trace = take(sizeof(unsigned long long) * 4 * ckv::kMaxCtas);
     w.st_tables = take(sizeof(int32_t) * (size_t)c.max_batch * c.max_pages_per_req);
     w.st_lens = take(sizeof(int32_t) * (size_t)c.max_batch);
     w.st_q = take((size_t)c.max_batch * c.num_q_heads * d2);
@@ -325,6 +326,7 @@ int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int
     ap.part_acc = pool->wsp<float>(pool->ws.part_acc);
     ap.part_ml = pool->wsp<float>(pool->ws.part_ml);
     ap.status = pool->wsp<uint32_t>(pool->ws.status);
+    ap.cta_trace = pool->wsp<unsigned long long>(pool->ws.cta_trace);
     ap.batch = batch;
     ap.max_pages_per_req = c.max_pages_per_req;
     ap.num_pages = c.num_pages;
@@ -484,6 +486,16 @@ int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch
     for (auto &e : ev) cudaEventDestroy(e);
     if (rc != CKV_OK) return rc;
     return kv_check_status(pool, stream, nullptr);
+}
+
+int32_t ckv_read_cta_trace(ckv_pool *pool, void *stream, uint64_t *h_trace)
+{
+    if (!pool || !h_trace) return fail(CKV_EINVAL, "ckv_read_cta_trace: NULL argument");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CKV_CUDA(cudaMemcpyAsync(h_trace, pool->d_ws + pool->ws.cta_trace, sizeof(uint64_t) * 4 * pool->num_ctas,
+                             cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaStreamSynchronize(s));
+    return CKV_OK;
 }
 
 int32_t ckv_profile_enable(ckv_pool *pool, int32_t enable)

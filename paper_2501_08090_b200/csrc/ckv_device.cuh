@@ -325,6 +325,7 @@ struct AttnParams {
     float *part_acc;                // [2*kMaxCtas][8][D]
     float *part_ml;                 // [2*kMaxCtas][16]  (m[8], l[8])
     uint32_t *status;
+    unsigned long long *cta_trace;  // [gridDim.x][4] ns: CTA start, first data consumed, producer done, consumers done
     int32_t batch, max_pages_per_req, num_pages, num_kv_heads, num_q_heads, group;
     int32_t layer_page_base;        // layer * num_pages
     float scale_log2;               // log2(e) / sqrt(d)
@@ -401,6 +402,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             mbar_init(empty_bar + s * 8, 1);
         }
         *abort_flag = 0;
+        p.cta_trace[blockIdx.x * 4 + 0] = global_timer_ns();
+        p.cta_trace[blockIdx.x * 4 + 1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -467,6 +470,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         }
         // Do not leave the CTA while copies into its shared memory may still be in flight.
         if (lane == 0) {
+            p.cta_trace[blockIdx.x * 4 + 2] = global_timer_ns();
             for (int k = max(0, it - S); k < it; ++k) {
                 const unsigned long long t0 = global_timer_ns();
                 while (!mbar_try_wait(full_bar + (k % S) * 8, (k / S) & 1)) {
@@ -530,6 +534,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 alive = __all_sync(0xffffffffu, alive);
             }
             if (!alive) continue;
+            if (it == 0 && lane == 0) p.cta_trace[blockIdx.x * 4 + 1] = global_timer_ns();
 
             const int ntok = min(kTileTokens, wk.L - ti * kTileTokens);     // valid tokens in this tile
             const bool full_tile = (ntok == kTileTokens);
@@ -690,6 +695,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         first_piece = false;
         wk.advance(p, n);
     }
+    if (threadIdx.x == 0) p.cta_trace[blockIdx.x * 4 + 3] = global_timer_ns();
 }
 
 // ------------------------------------------------------------------------------------------

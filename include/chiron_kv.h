@@ -109,7 +109,8 @@ int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch,
  *   out[r][h][:] = sum_j softmax_j( q[r][h].k_j / sqrt(d) ) v_j ,  j over request r's context,
  * computed as split-KV partials over balanced page ranges followed by a log-sum-exp combine.
  * d_q, d_out: bf16 [batch][num_q_heads][head_dim], 16-byte aligned; every row of d_out is
- * overwritten.  Enqueues a plan kernel, the attention kernel and the combine kernel.
+ * overwritten.  Enqueues ONE kernel: the partition is derived in its prologue and partials are
+ * merged by whichever warp finishes a (request, KV head) last.
  * Errors: CKV_EINVAL, CKV_ECUDA.
  */
 int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch,
@@ -117,22 +118,24 @@ int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch,
                          const void *d_q, void *d_out, void *stream);
 
 /*
- * The split-KV partition the next decode_attention would use for these lengths, copied to the
- * host for inspection (synchronises `stream`).  A "tile" is 64 consecutive tokens of one
- * (request, KV head); tiles are numbered request-major, then KV head, then position, and CTA c
- * owns tiles [c*tiles_per_cta, min((c+1)*tiles_per_cta, total_tiles)).
- *   h_header[4]   : total_tiles, tiles_per_cta, num_ctas (launched), num_ctas_with_work
- *   h_cta_start   : int32 [num_ctas][4] = request, kv head, first tile within that
- *                   (request, kv head), global index of the CTA's first tile; -1s if idle
- * h_cta_start must hold 4*ckv_get_partition() ints.  Errors: CKV_EINVAL, CKV_ECUDA.
+ * The split-KV partition decode_attention uses for these lengths, copied to the host for
+ * inspection (runs a small kernel and synchronises `stream`; decode_attention itself derives the
+ * same partition inside its attention kernel and launches no plan kernel).  A "tile" is 32
+ * consecutive tokens of one (request, KV head); tiles are numbered request-major, then KV head,
+ * then position, and span s -- the work of one warp -- owns tiles
+ * [s*tiles_per_span, min((s+1)*tiles_per_span, total_tiles)).
+ *   h_header[4]   : total_tiles, tiles_per_span, num_spans, num_spans_with_work
+ *   h_span_start  : int32 [num_spans][4] = request, kv head, first tile within that
+ *                   (request, kv head), global index of the span's first tile; -1s if idle
+ * h_span_start must hold 4*ckv_get_partition() ints.  Errors: CKV_EINVAL, CKV_ECUDA.
  */
 int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *stream,
-                    int32_t *h_header, int32_t *h_cta_start);
+                    int32_t *h_header, int32_t *h_span_start);
 
-/* Number of CTAs the partition is balanced over (default: one per SM).  Setting it changes
- * only how the context is split, never the result beyond fp32 summation order.
- * 1 <= num_ctas <= 1024.  Errors: CKV_EINVAL. */
-int32_t ckv_set_partition(ckv_pool *pool, int32_t num_ctas);
+/* Number of spans the partition is balanced over (default: warps per CTA x number of SMs).
+ * Setting it changes only how the context is split, never the result beyond fp32 summation
+ * order.  1 <= num_spans <= 2048.  Errors: CKV_EINVAL. */
+int32_t ckv_set_partition(ckv_pool *pool, int32_t num_spans);
 int32_t ckv_get_partition(const ckv_pool *pool);
 
 /* Synchronise `stream`, read and clear the device status word.  Returns CKV_OK, CKV_EBOUNDS
@@ -180,14 +183,15 @@ int32_t ckv_profile_enable(ckv_pool *pool, int32_t enable);
 int32_t ckv_profile_read(ckv_pool *pool, double *out_attention_ms, int32_t *out_launches);
 
 /*
- * Per-CTA timeline of the most recent attention kernel, for load-balance analysis (synchronises
+ * Per-span timeline of the most recent attention kernel, for load-balance analysis (synchronises
  * `stream`).  h_trace: uint64 [ckv_get_partition()][4], nanoseconds of the GPU's global timer:
- * CTA start, first tile consumed (0 if the CTA had no work), producer warp done, consumers done.
- * Errors: CKV_EINVAL, CKV_ECUDA.
+ * warp start, first tile landed (0 if the span had no work), last tile computed, span finished.
+ * h_span_start (may be NULL): int32 [ckv_get_partition()][4], the span starts the kernel derived
+ * itself, in decode_plan's format.  Errors: CKV_EINVAL, CKV_ECUDA.
  */
-int32_t ckv_read_cta_trace(ckv_pool *pool, void *stream, uint64_t *h_trace);
+int32_t ckv_read_span_trace(ckv_pool *pool, void *stream, uint64_t *h_trace, int32_t *h_span_start);
 
-/* Kernels launched through this handle since creation (append, plan, attention, combine). */
+/* Kernels launched through this handle since creation (append, attention, plan inspection). */
 int64_t ckv_launch_count(const ckv_pool *pool);
 
 /* Message describing the calling thread's most recent failure ("" if none). */

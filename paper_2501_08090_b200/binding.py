@@ -23,7 +23,7 @@ EXPORTS = (
     "kv_pool_bytes", "kv_workspace_bytes", "kv_pool_create", "kv_pool_destroy", "kv_append",
     "decode_attention", "decode_plan", "ckv_set_partition", "ckv_get_partition", "kv_check_status",
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
-    "ckv_launch_count", "ckv_last_error", "ckv_read_cta_trace",
+    "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace",
 )
 
 
@@ -64,7 +64,7 @@ def _load() -> ctypes.CDLL:
     lib.ckv_profile_enable.restype = i32; lib.ckv_profile_enable.argtypes = [vp, i32]
     lib.ckv_profile_read.restype = i32
     lib.ckv_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
-    lib.ckv_read_cta_trace.restype = i32; lib.ckv_read_cta_trace.argtypes = [vp, vp, vp]
+    lib.ckv_read_span_trace.restype = i32; lib.ckv_read_span_trace.argtypes = [vp, vp, vp, vp]
     lib.ckv_launch_count.restype = i64; lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_last_error.restype = ctypes.c_char_p; lib.ckv_last_error.argtypes = []
     return lib
@@ -167,17 +167,17 @@ class KvPool:
                                     _dev_ptr(out, torch.bfloat16), _stream_ptr(stream)))
 
     def decode_plan(self, seq_lens, stream=None):
-        """(header dict, int32 [num_ctas][4] array of span starts)."""
+        """(header dict, int32 [num_spans][4] array of span starts)."""
         batch = int(seq_lens.shape[0])
         header = np.zeros(4, dtype=np.int32)
         starts = np.zeros((self.get_partition(), 4), dtype=np.int32)
         _check(lib.decode_plan(self._h, batch, _dev_ptr(seq_lens, torch.int32), _stream_ptr(stream),
                                header.ctypes.data, starts.ctypes.data))
-        keys = ("total_tiles", "tiles_per_cta", "num_ctas", "ctas_with_work")
+        keys = ("total_tiles", "tiles_per_span", "num_spans", "spans_with_work")
         return dict(zip(keys, header.tolist())), starts
 
-    def set_partition(self, num_ctas: int) -> None:
-        _check(lib.ckv_set_partition(self._h, int(num_ctas)))
+    def set_partition(self, num_spans: int) -> None:
+        _check(lib.ckv_set_partition(self._h, int(num_spans)))
 
     def get_partition(self) -> int:
         return int(lib.ckv_get_partition(self._h))
@@ -226,11 +226,13 @@ class KvPool:
         _check(lib.ckv_profile_read(self._h, ctypes.byref(ms), ctypes.byref(n)))
         return float(ms.value), int(n.value)
 
-    def read_cta_trace(self, stream=None) -> np.ndarray:
-        """uint64 [num_ctas][4] ns: CTA start, first tile consumed, producer done, consumers done."""
+    def read_span_trace(self, stream=None):
+        """(uint64 [spans][4] ns: warp start, first tile landed, last tile computed, span finished;
+        int32 [spans][4] span starts as the attention kernel derived them)."""
         trace = np.zeros((self.get_partition(), 4), dtype=np.uint64)
-        _check(lib.ckv_read_cta_trace(self._h, _stream_ptr(stream), trace.ctypes.data))
-        return trace
+        starts = np.zeros((self.get_partition(), 4), dtype=np.int32)
+        _check(lib.ckv_read_span_trace(self._h, _stream_ptr(stream), trace.ctypes.data, starts.ctypes.data))
+        return trace, starts
 
     def launch_count(self) -> int:
         return int(lib.ckv_launch_count(self._h))

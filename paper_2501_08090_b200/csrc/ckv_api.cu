@@ -34,9 +34,9 @@ int32_t fail(int32_t code, const char *fmt, ...)
                         __FILE__, __LINE__);                                                  \
     } while (0)
 
-// Attention kernel shapes: ring depth is a multiple of the consumer-warp count (see the kernel).
-constexpr int kWarps128 = 6, kStages128 = 6;     // head_dim 128: 6 x 32 KB in flight per SM
-constexpr int kWarps64 = 4, kStages64 = 8;       // head_dim 64:  8 x 16 KB
+// Attention kernel shapes: warps per CTA (one CTA per SM) and ring stages per warp.
+constexpr int kWarps128 = 4, kStages128 = 3;     // head_dim 128: 4 warps x 3 stages x 16 KB = 192 KB per SM
+constexpr int kWarps64 = 4, kStages64 = 4;       // head_dim 64:  4 warps x 4 stages x 8 KB
 constexpr int kMaxProfile = 4096;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -66,7 +66,7 @@ bool config_ok(const ckv_config *c, const char **why)
 }
 
 struct WorkspaceLayout {
-    size_t status, header, cta_start, tile_prefix, part_acc, part_ml, cta_trace;
+    size_t status, header, span_start, part_acc, part_ml, arrivals, trace;
     size_t st_tables, st_lens, st_q, st_k, st_v, st_out;
     size_t total;
 };
@@ -79,11 +79,11 @@ WorkspaceLayout carve(const ckv_config &c)
     const size_t d2 = (size_t)c.head_dim * 2;
     w.status = take(256);
     w.header = take(sizeof(ckv::PlanHeader));
-    w.cta_start = take(sizeof(int4) * ckv::kMaxCtas);
-    w.tile_prefix = take(sizeof(int32_t) * ((size_t)c.max_batch + 1));
-    w.part_acc = take(sizeof(float) * 2 * ckv::kMaxCtas * ckv::kMaxGroup * c.head_dim);
-    w.part_ml = take(sizeof(float) * 2 * ckv::kMaxCtas * 2 * ckv::kMaxGroup);
-    w.cta_trace = take(sizeof(unsigned long long) * 4 * ckv::kMaxCtas);
+    w.span_start = take(sizeof(int4) * ckv::kMaxSpans);
+    w.part_acc = take(sizeof(float) * 2 * ckv::kMaxSpans * ckv::kMaxGroup * c.head_dim);
+    w.part_ml = take(sizeof(float) * 2 * ckv::kMaxSpans * 2 * ckv::kMaxGroup);
+    w.arrivals = take(sizeof(int32_t) * ckv::kMaxSpans);
+    w.trace = take(sizeof(unsigned long long) * 4 * ckv::kMaxSpans);
     w.st_tables = take(sizeof(int32_t) * (size_t)c.max_batch * c.max_pages_per_req);
     w.st_lens = take(sizeof(int32_t) * (size_t)c.max_batch);
     w.st_q = take((size_t)c.max_batch * c.num_q_heads * d2);
@@ -105,7 +105,7 @@ struct ckv_pool {
     ckv_config cfg;
     int device;
     int num_sms;
-    int num_ctas;                    // partition width
+    int num_spans;                   // partition width: one span per warp of the attention kernel
     uint8_t *d_pool;
     uint8_t *d_ws;
     WorkspaceLayout ws;
@@ -130,7 +130,8 @@ int32_t launch_attention(ckv_pool *pool, const ckv::AttnParams &ap, cudaStream_t
         CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
         configured_device = pool->device;
     }
-    kernel<<<pool->num_ctas, Lay::kThreads, Lay::kSmemBytes, stream>>>(pool->tmap, ap);
+    const int ctas = (pool->num_spans + W - 1) / W;
+    kernel<<<ctas, Lay::kThreads, Lay::kSmemBytes, stream>>>(pool->tmap, ap);
     CKV_CUDA(cudaGetLastError());
     return CKV_OK;
 }
@@ -147,22 +148,18 @@ int32_t check_call(ckv_pool *pool, int32_t layer, int32_t batch, const char *fn)
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-int32_t launch_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *d_out, cudaStream_t stream)
+int32_t launch_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, cudaStream_t stream)
 {
     const ckv_config &c = pool->cfg;
     ckv::PlanParams pp{};
     pp.seq_lens = d_seq_lens;
     pp.header = pool->wsp<ckv::PlanHeader>(pool->ws.header);
-    pp.cta_start = pool->wsp<int4>(pool->ws.cta_start);
-    pp.tile_prefix = pool->wsp<int32_t>(pool->ws.tile_prefix);
-    pp.status = pool->wsp<uint32_t>(pool->ws.status);
-    pp.out = static_cast<uint16_t *>(d_out);
+    pp.span_start = pool->wsp<int4>(pool->ws.span_start);
     pp.batch = batch;
     pp.max_pages_per_req = c.max_pages_per_req;
     pp.num_kv_heads = c.num_kv_heads;
-    pp.num_ctas = pool->num_ctas;
-    pp.out_row_elems = c.num_q_heads * c.head_dim;
-    ckv::splitkv_plan_kernel<<<1, ckv::kPlanThreads, sizeof(int32_t) * ((size_t)batch + 1), stream>>>(pp);
+    pp.num_spans = pool->num_spans;
+    ckv::splitkv_plan_kernel<<<(pool->num_spans + 7) / 8, 256, 0, stream>>>(pp);
     CKV_CUDA(cudaGetLastError());
     pool->launches += 1;
     return CKV_OK;
@@ -214,7 +211,7 @@ int32_t kv_pool_create(const ckv_config *cfg, void *d_pool, size_t pool_bytes, v
     p->cfg = *cfg;
     p->device = device;
     p->num_sms = sms;
-    p->num_ctas = std::min(sms, ckv::kMaxCtas);
+    p->num_spans = std::min(sms * (cfg->head_dim == 128 ? kWarps128 : kWarps64), ckv::kMaxSpans);
     p->d_pool = static_cast<uint8_t *>(d_pool);
     p->d_ws = static_cast<uint8_t *>(d_workspace);
     p->ws = ws;
@@ -264,15 +261,15 @@ int32_t kv_pool_destroy(ckv_pool *pool)
     return CKV_OK;
 }
 
-int32_t ckv_set_partition(ckv_pool *pool, int32_t num_ctas)
+int32_t ckv_set_partition(ckv_pool *pool, int32_t num_spans)
 {
     if (!pool) return fail(CKV_EINVAL, "ckv_set_partition: pool is NULL");
-    if (num_ctas < 1 || num_ctas > ckv::kMaxCtas) return fail(CKV_EINVAL, "ckv_set_partition: %d outside [1, %d]", num_ctas, ckv::kMaxCtas);
-    pool->num_ctas = num_ctas;
+    if (num_spans < 1 || num_spans > ckv::kMaxSpans) return fail(CKV_EINVAL, "ckv_set_partition: %d outside [1, %d]", num_spans, ckv::kMaxSpans);
+    pool->num_spans = num_spans;
     return CKV_OK;
 }
 
-int32_t ckv_get_partition(const ckv_pool *pool) { return pool ? pool->num_ctas : CKV_EINVAL; }
+int32_t ckv_get_partition(const ckv_pool *pool) { return pool ? pool->num_spans : CKV_EINVAL; }
 
 int64_t ckv_launch_count(const ckv_pool *pool) { return pool ? pool->launches : 0; }
 
@@ -314,19 +311,17 @@ int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int
     const ckv_config &c = pool->cfg;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
-    if (int32_t rc = launch_plan(pool, batch, d_seq_lens, d_out, s)) return rc;
-
     ckv::AttnParams ap{};
     ap.block_tables = d_block_tables;
     ap.seq_lens = d_seq_lens;
     ap.q = static_cast<const uint16_t *>(d_q);
     ap.out = static_cast<uint16_t *>(d_out);
-    ap.header = pool->wsp<ckv::PlanHeader>(pool->ws.header);
-    ap.cta_start = pool->wsp<int4>(pool->ws.cta_start);
     ap.part_acc = pool->wsp<float>(pool->ws.part_acc);
     ap.part_ml = pool->wsp<float>(pool->ws.part_ml);
+    ap.arrivals = pool->wsp<int32_t>(pool->ws.arrivals);
+    ap.span_start = pool->wsp<int4>(pool->ws.span_start);
+    ap.trace = pool->wsp<unsigned long long>(pool->ws.trace);
     ap.status = pool->wsp<uint32_t>(pool->ws.status);
-    ap.cta_trace = pool->wsp<unsigned long long>(pool->ws.cta_trace);
     ap.batch = batch;
     ap.max_pages_per_req = c.max_pages_per_req;
     ap.num_pages = c.num_pages;
@@ -334,6 +329,7 @@ int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int
     ap.num_q_heads = c.num_q_heads;
     ap.group = c.num_q_heads / c.num_kv_heads;
     ap.layer_page_base = layer * c.num_pages;
+    ap.num_spans = pool->num_spans;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
 
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -356,35 +352,18 @@ int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int
     if (rc) return rc;
     if (ev1) CKV_CUDA(cudaEventRecord(ev1, s));
     pool->launches += 1;
-
-    if (pool->num_ctas > 1) {
-        ckv::CombineParams cp{};
-        cp.header = ap.header;
-        cp.tile_prefix = pool->wsp<int32_t>(pool->ws.tile_prefix);
-        cp.part_acc = ap.part_acc;
-        cp.part_ml = ap.part_ml;
-        cp.out = ap.out;
-        cp.batch = batch;
-        cp.num_kv_heads = c.num_kv_heads;
-        cp.num_q_heads = c.num_q_heads;
-        cp.group = ap.group;
-        cp.head_dim = c.head_dim;
-        ckv::lse_combine_kernel<<<pool->num_ctas - 1, 256, 0, s>>>(cp);
-        CKV_CUDA(cudaGetLastError());
-        pool->launches += 1;
-    }
     return CKV_OK;
 }
 
 int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *stream,
-                    int32_t *h_header, int32_t *h_cta_start)
+                    int32_t *h_header, int32_t *h_span_start)
 {
     if (int32_t rc = check_call(pool, 0, batch, "decode_plan")) return rc;
-    if (!d_seq_lens || !h_header || !h_cta_start) return fail(CKV_EINVAL, "decode_plan: NULL argument");
+    if (!d_seq_lens || !h_header || !h_span_start) return fail(CKV_EINVAL, "decode_plan: NULL argument");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (int32_t rc = launch_plan(pool, batch, d_seq_lens, nullptr, s)) return rc;
+    if (int32_t rc = launch_plan(pool, batch, d_seq_lens, s)) return rc;
     CKV_CUDA(cudaMemcpyAsync(h_header, pool->d_ws + pool->ws.header, sizeof(ckv::PlanHeader), cudaMemcpyDeviceToHost, s));
-    CKV_CUDA(cudaMemcpyAsync(h_cta_start, pool->d_ws + pool->ws.cta_start, sizeof(int4) * pool->num_ctas, cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaMemcpyAsync(h_span_start, pool->d_ws + pool->ws.span_start, sizeof(int4) * pool->num_spans, cudaMemcpyDeviceToHost, s));
     CKV_CUDA(cudaStreamSynchronize(s));
     return CKV_OK;
 }
@@ -398,6 +377,11 @@ int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits)
     CKV_CUDA(cudaMemsetAsync(pool->d_ws + pool->ws.status, 0, sizeof bits, s));
     CKV_CUDA(cudaStreamSynchronize(s));
     if (out_bits) *out_bits = bits;
+    if (bits & ckv::kStatusWaitLimit) {
+        // a warp that gave up may have left arrival counters half-way; start the next launch clean
+        CKV_CUDA(cudaMemsetAsync(pool->d_ws + pool->ws.arrivals, 0, sizeof(int32_t) * ckv::kMaxSpans, s));
+        CKV_CUDA(cudaStreamSynchronize(s));
+    }
     if (bits & ckv::kStatusWaitLimit) return fail(CKV_ETIMEOUT, "device status 0x%x: a bounded wait gave up", bits);
     if (bits & (ckv::kStatusBadLength | ckv::kStatusBadPage))
         return fail(CKV_EBOUNDS, "device status 0x%x: %s%s", bits, (bits & ckv::kStatusBadLength) ? "[context length out of range]" : "",
@@ -488,12 +472,15 @@ int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch
     return kv_check_status(pool, stream, nullptr);
 }
 
-int32_t ckv_read_cta_trace(ckv_pool *pool, void *stream, uint64_t *h_trace)
+int32_t ckv_read_span_trace(ckv_pool *pool, void *stream, uint64_t *h_trace, int32_t *h_span_start)
 {
-    if (!pool || !h_trace) return fail(CKV_EINVAL, "ckv_read_cta_trace: NULL argument");
+    if (!pool || !h_trace) return fail(CKV_EINVAL, "ckv_read_span_trace: NULL argument");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    CKV_CUDA(cudaMemcpyAsync(h_trace, pool->d_ws + pool->ws.cta_trace, sizeof(uint64_t) * 4 * pool->num_ctas,
+    CKV_CUDA(cudaMemcpyAsync(h_trace, pool->d_ws + pool->ws.trace, sizeof(uint64_t) * 4 * pool->num_spans,
                              cudaMemcpyDeviceToHost, s));
+    if (h_span_start)
+        CKV_CUDA(cudaMemcpyAsync(h_span_start, pool->d_ws + pool->ws.span_start, sizeof(int4) * pool->num_spans,
+                                 cudaMemcpyDeviceToHost, s));
     CKV_CUDA(cudaStreamSynchronize(s));
     return CKV_OK;
 }

@@ -1,5 +1,5 @@
 // Device code of the decode-iteration hot path for sm_100a: KV append, split-KV plan,
-// paged grouped-query partial attention (TMA-fed, tensor-core) and the log-sum-exp combine.
+// paged grouped-query partial attention (TMA-fed, tensor-core) with its log-sum-exp combine.
 //
 // Pool layout (bf16): [layer][page][kv_head][K|V][slot 0..15][d]  -- one (page, kv_head) is a
 // contiguous block of 32 rows (16 key rows, then 16 value rows) of d elements.
@@ -12,10 +12,10 @@
 namespace ckv {
 
 constexpr int kPageSize = 16;        // tokens per page
-constexpr int kPagesPerTile = 4;     // a tile is the scheduling unit: 64 tokens of one (request, kv head)
+constexpr int kPagesPerTile = 2;     // a tile is the scheduling unit: 32 tokens of one (request, kv head)
 constexpr int kTileTokens = kPageSize * kPagesPerTile;
 constexpr int kMaxGroup = 8;         // query heads per KV head handled by one MMA column block
-constexpr int kMaxCtas = 1024;       // upper bound on the partition width
+constexpr int kMaxSpans = 2048;      // upper bound on the partition width (one span per warp)
 constexpr int kMaxBatch = 8192;
 
 constexpr uint32_t kStatusBadLength = 1u;
@@ -24,11 +24,13 @@ constexpr uint32_t kStatusWaitLimit = 4u;
 
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // bound of every device-side wait
 
+// The split-KV partition.  Tiles of all (request, kv head) pairs are numbered request-major, then
+// kv head, then position; span s owns tiles [s*q, min((s+1)*q, total)) with q = ceil(total/spans).
 struct PlanHeader {
-    int32_t total_tiles;      // over all (request, kv head)
-    int32_t tiles_per_cta;    // span length q: CTA c owns tiles [c*q, min((c+1)*q, total))
-    int32_t num_ctas;         // partition width
-    int32_t ctas_with_work;
+    int32_t total_tiles;
+    int32_t tiles_per_span;
+    int32_t num_spans;
+    int32_t spans_with_work;
 };
 
 // A context length is usable if 1 <= L <= table capacity; otherwise the request has no tiles.
@@ -84,96 +86,102 @@ __global__ void kv_append_kernel(const AppendParams p)
 }
 
 // ------------------------------------------------------------------------------------------
-// K2: split-KV plan.  One CTA: per-request tile counts, their exclusive prefix sum, the span
-// length, and for every CTA of the partition the (request, kv head, tile) its span starts at.
+// K2: the split-KV plan.
+//
+// The attention kernel derives its partition from seq_lens in its own prologue (warp_plan below),
+// so a decode step launches no separate plan kernel.  splitkv_plan_kernel computes the same
+// partition for every span at once, for inspection through decode_plan().
 // ------------------------------------------------------------------------------------------
+struct SpanStart {
+    int r, h, tile;        // first tile of the span: request, kv head, tile within (r, h); r = -1: no work
+    int tiles_r;           // tiles per kv head of request r
+    int L;                 // context length of request r
+    int count;             // tiles in the span
+    int begin;             // global index of the span's first tile
+    int total, q;          // header values
+};
+
+// Executed by one whole warp.  Two passes over seq_lens: the total, then the request that holds
+// tile span*q.  If `zero_rows` is set (one warp of the grid), requests with an unusable length
+// get their output rows cleared and the status word flagged.
+__device__ __forceinline__ SpanStart warp_plan(const int32_t *__restrict__ seq_lens, int batch, int max_pages_per_req,
+                                               int num_kv_heads, int num_spans, int span, int lane,
+                                               uint16_t *zero_rows, int out_row_elems, uint32_t *status)
+{
+    SpanStart s;
+    int sum = 0;
+    for (int base = 0; base < batch; base += 32) {
+        const int r = base + lane;
+        if (r < batch) {
+            const int t = tiles_of_length(__ldg(seq_lens + r), max_pages_per_req);
+            sum += t;
+            if (t == 0 && zero_rows != nullptr) {
+                atomicOr(status, kStatusBadLength);
+                for (int i = 0; i < out_row_elems; ++i) zero_rows[(size_t)r * out_row_elems + i] = 0;
+            }
+        }
+    }
+#pragma unroll
+    for (int x = 16; x > 0; x >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, x);
+    s.total = sum * num_kv_heads;
+    s.q = max(1, (s.total + num_spans - 1) / num_spans);
+    const long long begin = (long long)span * s.q;
+    s.r = -1; s.h = s.tile = s.tiles_r = s.L = s.count = 0;
+    s.begin = (int)min(begin, (long long)s.total);
+    if (begin >= s.total) return s;
+    s.count = (int)min((long long)s.q, (long long)s.total - begin);
+
+    long long running = 0;                               // tiles (all heads) before request `base`
+    for (int base = 0; base < batch; base += 32) {
+        const int r = base + lane;
+        const int L = r < batch ? __ldg(seq_lens + r) : 0;
+        const int t = r < batch ? tiles_of_length(L, max_pages_per_req) : 0;
+        int incl = t;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const long long upto = running + (long long)incl * num_kv_heads;     // tiles through request r
+        const unsigned hit = __ballot_sync(0xffffffffu, upto > begin);
+        if (hit) {
+            const int src = __ffs(hit) - 1;
+            const int t_r = __shfl_sync(0xffffffffu, t, src);
+            const int L_r = __shfl_sync(0xffffffffu, L, src);
+            const long long before = __shfl_sync(0xffffffffu, upto, src) - (long long)t_r * num_kv_heads;
+            const int rem = (int)(begin - before);
+            s.r = base + src; s.tiles_r = t_r; s.L = L_r;
+            s.h = rem / t_r; s.tile = rem % t_r;
+            return s;
+        }
+        running = __shfl_sync(0xffffffffu, upto, 31);
+    }
+    return s;                                            // not reached: begin < total
+}
+
 struct PlanParams {
     const int32_t *seq_lens;
     PlanHeader *header;
-    int4 *cta_start;                // [num_ctas]
-    int32_t *tile_prefix;           // [batch + 1], tiles per KV head before request r
-    uint32_t *status;
-    uint16_t *out;                  // rows of requests with an unusable length are zero-filled
-    int32_t batch, max_pages_per_req, num_kv_heads, num_ctas, out_row_elems;
+    int4 *span_start;               // [num_spans] request, kv head, tile, global tile index (-1s if idle)
+    int32_t batch, max_pages_per_req, num_kv_heads, num_spans;
 };
 
-constexpr int kPlanThreads = 1024;
-
-__global__ void __launch_bounds__(kPlanThreads) splitkv_plan_kernel(const PlanParams p)
+__global__ void splitkv_plan_kernel(const PlanParams p)
 {
-    extern __shared__ int32_t s_prefix[];        // [batch + 1]
-    __shared__ int32_t s_warp[32];
-    const int tid = threadIdx.x;
-    const int per = (p.batch + kPlanThreads - 1) / kPlanThreads;
-    const int r0 = tid * per;
-    const int r1 = min(p.batch, r0 + per);
-
-    int local = 0;
-    for (int r = r0; r < r1; ++r) {
-        const int t = tiles_of_length(p.seq_lens[r], p.max_pages_per_req);
-        if (t == 0) {
-            atomicOr(p.status, kStatusBadLength);
-            if (p.out != nullptr)
-                for (int i = 0; i < p.out_row_elems; ++i) p.out[(size_t)r * p.out_row_elems + i] = 0;
-        }
-        s_prefix[r] = t;                          // overwritten by the prefix below
-        local += t;
-    }
-    // exclusive scan of the per-thread sums
-    int incl = local;
-    const int lane = tid & 31, warp = tid >> 5;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        int w = s_warp[lane];
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, w, o);
-            if (lane >= o) w += v;
-        }
-        s_warp[lane] = w;                         // inclusive over warps
-    }
-    __syncthreads();
-    int run = incl - local + (warp > 0 ? s_warp[warp - 1] : 0);
-    for (int r = r0; r < r1; ++r) {
-        const int t = s_prefix[r];
-        s_prefix[r] = run;
-        run += t;
-    }
-    if (tid == kPlanThreads - 1) s_prefix[p.batch] = s_warp[31];
-    __syncthreads();
-
-    const int per_head_total = s_prefix[p.batch];
-    const int total = per_head_total * p.num_kv_heads;
-    const int q = max(1, (total + p.num_ctas - 1) / p.num_ctas);
-    for (int r = tid; r <= p.batch; r += kPlanThreads) p.tile_prefix[r] = s_prefix[r];
-    if (tid == 0) {
-        p.header->total_tiles = total;
-        p.header->tiles_per_cta = q;
-        p.header->num_ctas = p.num_ctas;
-        p.header->ctas_with_work = (total + q - 1) / q;
-    }
-    for (int c = tid; c < p.num_ctas; c += kPlanThreads) {
-        const long long t0 = (long long)c * q;
-        int4 st = make_int4(-1, -1, -1, -1);
-        if (t0 < total) {
-            // smallest r' with Hkv*prefix[r'] > t0; the span starts inside request r' - 1
-            int lo = 0, hi = p.batch;             // prefix[0] = 0 <= t0 < Hkv*prefix[batch]
-            while (hi - lo > 1) {
-                const int mid = (lo + hi) >> 1;
-                if ((long long)s_prefix[mid] * p.num_kv_heads > t0) hi = mid; else lo = mid;
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int span = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; span < p.num_spans; span += warps) {
+        const SpanStart s = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span,
+                                      lane, nullptr, 0, nullptr);
+        if (lane == 0) {
+            p.span_start[span] = s.r < 0 ? make_int4(-1, -1, -1, -1) : make_int4(s.r, s.h, s.tile, s.begin);
+            if (span == 0) {
+                p.header->total_tiles = s.total;
+                p.header->tiles_per_span = s.q;
+                p.header->num_spans = p.num_spans;
+                p.header->spans_with_work = (s.total + s.q - 1) / s.q;
             }
-            const int r = lo;
-            const int tr = s_prefix[r + 1] - s_prefix[r];
-            const int rem = (int)(t0 - (long long)s_prefix[r] * p.num_kv_heads);
-            st = make_int4(r, rem / tr, rem % tr, (int)t0);
         }
-        p.cta_start[c] = st;
     }
 }
 
@@ -202,11 +210,6 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 {
     uint32_t done;
@@ -218,18 +221,15 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return done;
 }
 
-// Wait for a phase of an mbarrier, giving up after kWaitLimitNs or as soon as another thread of
-// the CTA has given up.  Returns false when it gave up (the caller then skips its work).
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                                  uint32_t *status)
+// Wait for a phase of an mbarrier, giving up after kWaitLimitNs.  Returns false when it gave up;
+// the status word is flagged and the caller stops working.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t *status)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
         if (global_timer_ns() - t0 > kWaitLimitNs) {
-            *abort_flag = 1;
             atomicOr(status, kStatusWaitLimit);
             return false;
         }
@@ -241,6 +241,11 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void fence_proxy_async()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
@@ -285,53 +290,59 @@ __device__ __forceinline__ float fast_exp2(float x)
     return y;
 }
 
-__device__ __forceinline__ void named_barrier_sync(int id, int threads)
+__device__ __forceinline__ float ld_cg_f32(const float *p)
 {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+    float v;
+    asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
 }
 
-__device__ __forceinline__ uint16_t f32_to_bf16_rn(float x)
+__device__ __forceinline__ float4 ld_cg_f32x4(const float *p)
 {
-    uint16_t h;
-    asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(x));
-    return h;
+    float4 v;
+    asm volatile("ld.global.cg.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
 }
 
 // ------------------------------------------------------------------------------------------
-// K3: paged partial attention.
+// K3 + K4: paged partial attention with the log-sum-exp combine folded in.
 //
-// One persistent CTA per span of the plan.  Warp W (the last) is the producer: it walks the
-// span tile by tile, looks the pages up in the block table and issues one TMA box load per
-// 128-byte column block of each (page, kv head) into a ring of S stages (one stage = one tile =
-// up to 4 pages).  Warps 0..W-1 are consumers; stage number `it` of the CTA is consumed by warp
-// it % W, which keeps its own running maximum m, sum l and accumulator O for the current
-// (request, kv head) piece.  At the end of a piece the consumer warps merge their states through
-// shared memory and write either the final bf16 output row (the piece covered the whole
-// context) or an fp32 partial (m, l, O) for the combine kernel.
+// Every WARP is an independent worker: it owns one span of the plan, a private ring of NS stages
+// in shared memory with one mbarrier per stage, and a small staging tile.  A stage holds one tile
+// (2 pages: 32 key rows and 32 value rows of one kv head).  The warp itself issues the TMA box
+// loads of the tile NS stages ahead of the one it computes on (an "issue" cursor and a "compute"
+// cursor walk the same span), so there is no producer warp, no cross-warp merge and no CTA-wide
+// barrier anywhere; a CTA is just W such warps sharing an SM's shared memory.
 //
 // MMA formulation (operands swapped so the tile's tokens fill the M dimension):
 //   S^T[tok 16 x g 8]  = K[tok 16 x d] . Q^T[d x g 8]          (A = K rows via ldmatrix)
 //   O^T[d 16 x g 8]   += V^T[d 16 x tok 16] . P^T[tok 16 x g 8] (A = V via ldmatrix.trans)
 // The S^T accumulator fragment holds (token = lane/4 [+8], g = 2*(lane%4)+{0,1}); packed to bf16
 // and transposed with movmatrix it is exactly the B fragment of P^T.
+//
+// A piece is the part of one (request, kv head) that falls inside the span.  When it covers the
+// whole context the warp normalises and writes the bf16 output rows itself.  Otherwise it stores
+// an fp32 partial (m, l, O) and bumps an arrival counter; whichever warp arrives last for that
+// (request, kv head) merges all its partials (wait-free: nobody ever waits for another warp).
 // ------------------------------------------------------------------------------------------
 struct AttnParams {
     const int32_t *block_tables;
     const int32_t *seq_lens;
     const uint16_t *q;
     uint16_t *out;
-    const PlanHeader *header;
-    const int4 *cta_start;
-    float *part_acc;                // [2*kMaxCtas][8][D]
-    float *part_ml;                 // [2*kMaxCtas][16]  (m[8], l[8])
+    float *part_acc;                // [2*kMaxSpans][8][D]
+    float *part_ml;                 // [2*kMaxSpans][16]  (m[8], l[8])
+    int32_t *arrivals;              // [kMaxSpans], all zero between launches
+    int4 *span_start;               // [kMaxSpans] what each span started at (diagnostic)
+    unsigned long long *trace;      // [kMaxSpans][4] ns: start, first tile landed, last tile done, span done
     uint32_t *status;
-    unsigned long long *cta_trace;  // [gridDim.x][4] ns: CTA start, first data consumed, producer done, consumers done
     int32_t batch, max_pages_per_req, num_pages, num_kv_heads, num_q_heads, group;
     int32_t layer_page_base;        // layer * num_pages
+    int32_t num_spans;
     float scale_log2;               // log2(e) / sqrt(d)
 };
 
-template <int D, int W, int S>
+template <int D, int W, int NS>
 struct AttnLayout {
     static constexpr int kHalves = D / 64;                       // 128-byte column blocks per row
     static constexpr int kHalfBytes = 32 * 128;                  // one TMA box: 32 rows x 128 B
@@ -339,158 +350,156 @@ struct AttnLayout {
     static constexpr int kStageBytes = kPagesPerTile * kPageBytes;
     static constexpr int kKSteps = D / 16;
     static constexpr int kDTiles = D / 16;
-    static constexpr int kScratchFloats = W * D * kMaxGroup + W * 2 * kMaxGroup;
-    static constexpr int kSmemBytes = S * kStageBytes + kScratchFloats * 4 + 2 * S * 8 + 16 + 1024;
-    static constexpr int kThreads = (W + 1) * 32;
+    static constexpr int kStagePitch = D + 4;                    // floats per staging row (bank spread)
+    static constexpr int kStagingBytes = kMaxGroup * kStagePitch * 4;
+    static constexpr int kRingBytes = W * NS * kStageBytes;
+    static constexpr int kSmemBytes = kRingBytes + W * kStagingBytes + W * NS * 8 + 1024;
+    static constexpr int kThreads = W * 32;
 };
 
-// Position of a CTA inside its span; producer and consumers advance identical copies.
-struct SpanWalk {
-    int r, h, tile;       // next tile to process: request, kv head, tile within (r, h)
-    int remaining;        // tiles left in the span
+// A cursor over the tiles of a span.  The issue cursor and the compute cursor are two copies.
+struct SpanCursor {
+    int r, h, tile;       // next tile: request, kv head, tile within (r, h)
     int L, tiles;         // length and tile count of request r
 
-    __device__ __forceinline__ void load_request(const AttnParams &p)
+    // step to the next tile; returns false when it left the last request
+    __device__ __forceinline__ bool next(const AttnParams &p)
     {
-        L = p.seq_lens[r];
-        tiles = tiles_of_length(L, p.max_pages_per_req);
-    }
-    // tiles of the current piece
-    __device__ __forceinline__ int piece_tiles() const { return min(tiles - tile, remaining); }
-    // move past the current piece to the start of the next (request, kv head)
-    __device__ __forceinline__ void advance(const AttnParams &p, int n)
-    {
-        remaining -= n;
-        if (remaining <= 0) return;
+        if (++tile < tiles) return true;
         tile = 0;
-        if (++h == p.num_kv_heads) {
-            h = 0;
-            do {
-                if (++r >= p.batch) { remaining = 0; return; }
-                load_request(p);
-            } while (tiles == 0);
-        }
+        if (++h < p.num_kv_heads) return true;
+        h = 0;
+        do {
+            if (++r >= p.batch) return false;
+            L = __ldg(p.seq_lens + r);
+            tiles = tiles_of_length(L, p.max_pages_per_req);
+        } while (tiles == 0);
+        return true;
     }
 };
 
-template <int D, int W, int S>
-__global__ void __launch_bounds__((W + 1) * 32, 1)
+template <int D, int W, int NS>
+__global__ void __launch_bounds__(W * 32, 1)
 paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnParams p)
 {
-    using Lay = AttnLayout<D, W, S>;
-    // Stage `it` lives in slot it % S and is consumed by warp it % W.  A consumer tells "my data
-    // has landed" from the parity of the slot's barrier, which is only unambiguous if it cannot
-    // get a whole phase ahead of the slot's previous use.  Copies complete out of order, so that
-    // holds only when the previous use of the slot was consumed by the SAME warp: S % W == 0.
-    static_assert(S % W == 0, "every ring slot must always be consumed by the same warp");
+    using Lay = AttnLayout<D, W, NS>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    float *scratch_o = (float *)(smem + S * Lay::kStageBytes);            // [W][D][8]
-    float *scratch_ml = scratch_o + W * D * kMaxGroup;                     // [W][16]
-    uint64_t *bars = (uint64_t *)(scratch_ml + W * 2 * kMaxGroup);         // full[S], empty[S]
-    volatile int *abort_flag = (volatile int *)(bars + 2 * S);
-
-    const uint32_t stage_base = smem_u32(smem);
-    const uint32_t full_bar = smem_u32(bars);
-    const uint32_t empty_bar = full_bar + S * 8;
-
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int span = blockIdx.x * W + warp;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(full_bar + s * 8, 1);
-            mbar_init(empty_bar + s * 8, 1);
-        }
-        *abort_flag = 0;
-        p.cta_trace[blockIdx.x * 4 + 0] = global_timer_ns();
-        p.cta_trace[blockIdx.x * 4 + 1] = 0;
+    const uint32_t ring = smem_u32(smem) + warp * NS * Lay::kStageBytes;
+    float *staging = (float *)(smem + Lay::kRingBytes + warp * Lay::kStagingBytes);
+    const uint32_t bars = smem_u32(smem + Lay::kRingBytes + W * Lay::kStagingBytes) + warp * NS * 8;
+
+    if (span >= p.num_spans) return;
+    unsigned long long t_start = 0;
+    if (lane == 0) {
+        t_start = global_timer_ns();
+        for (int s = 0; s < NS; ++s) mbar_init(bars + s * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fence_proxy_async();
     }
-    __syncthreads();
+    __syncwarp();
 
-    const int total = p.header->total_tiles;
-    const int q_span = p.header->tiles_per_cta;
-    const long long span_begin = (long long)blockIdx.x * q_span;
-    if (span_begin >= total) return;
-    const int4 st = p.cta_start[blockIdx.x];
-
-    SpanWalk wk;
-    wk.r = st.x; wk.h = st.y; wk.tile = st.z;
-    wk.remaining = (int)min((long long)q_span, (long long)total - span_begin);
-    wk.load_request(p);
-
-    if (warp == W) {
-        // ------------------------------------------------------------------ producer warp
-        int it = 0;
-        bool ok = true;
-        int pf_val = -1, pf_row = -1;              // chunk 0 of the row the next piece is expected in
-        while (wk.remaining > 0 && ok) {
-            const int n = wk.piece_tiles();
-            const int n_pages = (wk.L + kPageSize - 1) / kPageSize;
-            const int32_t *row = p.block_tables + (size_t)wk.r * p.max_pages_per_req;
-            auto load_chunk = [&](const int32_t *rw, int chunk) -> int {
-                const int idx = chunk * 32 + lane;
-                return idx < p.max_pages_per_req ? __ldg(rw + idx) : -1;
-            };
-            int cur_chunk = wk.tile / 8;
-            int cur_val = (cur_chunk == 0 && pf_row == wk.r) ? pf_val : load_chunk(row, cur_chunk);
-            int nxt_val = load_chunk(row, cur_chunk + 1);
-            // the next piece starts at tile 0 of this row (next kv head) or of the next request
-            pf_row = (wk.h + 1 < p.num_kv_heads) ? wk.r : wk.r + 1;
-            pf_val = (pf_row < p.batch) ? load_chunk(p.block_tables + (size_t)pf_row * p.max_pages_per_req, 0) : -1;
-
-            for (int ti = wk.tile; ti < wk.tile + n && ok; ++ti, ++it) {
-                const int ck = ti / 8;
-                if (ck != cur_chunk) {
-                    cur_chunk = ck;
-                    cur_val = nxt_val;
-                    nxt_val = load_chunk(row, ck + 1);
-                }
-                const int np = min(kPagesPerTile, n_pages - ti * kPagesPerTile);
-                const int pg = lane / Lay::kHalves, hf = lane % Lay::kHalves;
-                int page = __shfl_sync(0xffffffffu, cur_val, ((ti & 7) * kPagesPerTile + pg) & 31);
-                const int slot = it % S;
-                ok = mbar_wait_bounded(empty_bar + slot * 8, ((it / S) & 1) ^ 1, abort_flag, p.status);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                if (lane == 0) mbar_arrive_expect_tx(full_bar + slot * 8, np * Lay::kPageBytes);
-                __syncwarp();
-                if (lane < np * Lay::kHalves) {
-                    if (page < 0 || page >= p.num_pages) {
-                        atomicOr(p.status, kStatusBadPage);
-                        page = 0;
-                    }
-                    const int y = ((p.layer_page_base + page) * p.num_kv_heads + wk.h) * 32;
-                    tma_load_2d(stage_base + slot * Lay::kStageBytes + pg * Lay::kPageBytes + hf * Lay::kHalfBytes,
-                                &tmap, hf * 64, y, full_bar + slot * 8);
-                }
-            }
-            wk.advance(p, n);
-        }
-        // Do not leave the CTA while copies into its shared memory may still be in flight.
-        if (lane == 0) {
-            p.cta_trace[blockIdx.x * 4 + 2] = global_timer_ns();
-            for (int k = max(0, it - S); k < it; ++k) {
-                const unsigned long long t0 = global_timer_ns();
-                while (!mbar_try_wait(full_bar + (k % S) * 8, (k / S) & 1)) {
-                    if (global_timer_ns() - t0 > kWaitLimitNs) {
-                        atomicOr(p.status, kStatusWaitLimit);
-                        break;
-                    }
-                }
-            }
-        }
+    // ---- plan: where does this warp's span start?
+    const SpanStart st = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane,
+                                   span == 0 ? p.out : nullptr, p.num_q_heads * D, p.status);
+    if (lane == 0) {
+        p.span_start[span] = st.r < 0 ? make_int4(-1, -1, -1, -1) : make_int4(st.r, st.h, st.tile, st.begin);
+        p.trace[span * 4 + 0] = t_start;
+        p.trace[span * 4 + 1] = 0;
+    }
+    if (st.r < 0) {
+        if (lane == 0) p.trace[span * 4 + 2] = p.trace[span * 4 + 3] = global_timer_ns();
         return;
     }
-
-    // ---------------------------------------------------------------------- consumer warps
-    const int g_row = lane >> 2;                 // query head (within the group) this lane loads Q for
-    const int g0 = (lane & 3) * 2;               // first of the two group columns this lane accumulates
+    const int n_total = st.count;
+    const int q_span = st.q;
     const int G = p.group;
 
-    // ldmatrix lane offsets inside one page block (without the column-block and page terms)
-    uint32_t k_off[4], v_off[4];
+    // ---- issue side: block-table entries travel in registers, 32 pages (16 tiles) per chunk
+    SpanCursor ic;
+    ic.r = st.r; ic.h = st.h; ic.tile = st.tile; ic.L = st.L; ic.tiles = st.tiles_r;
+    int issued = 0;
+    bool alive = true;
+    auto table_row = [&](int r) { return p.block_tables + (size_t)r * p.max_pages_per_req; };
+    auto load_chunk = [&](int r, int chunk) -> int {
+        const int idx = chunk * 32 + lane;
+        return (r < p.batch && idx < p.max_pages_per_req) ? __ldg(table_row(r) + idx) : -1;
+    };
+    constexpr int kTilesPerChunk = 32 / kPagesPerTile;
+    int cur_chunk = ic.tile / kTilesPerChunk;
+    int cur_val = load_chunk(ic.r, cur_chunk);
+    int nxt_val = load_chunk(ic.r, cur_chunk + 1);
+    // chunk 0 of the row the NEXT (request, kv head) will read: this row again, or the next request's
+    int pf_row = (ic.h + 1 < p.num_kv_heads) ? ic.r : ic.r + 1;
+    int pf_val = load_chunk(pf_row, 0);
+
+    // query fragments of a (request, kv head), fetched when the issue cursor enters it
+    uint32_t qn[Lay::kKSteps][2];
+    int qn_r = -1, qn_h = -1;
+    const int g_row = lane >> 2;                 // query head (within the group) this lane loads Q for
+    auto load_q = [&](uint32_t (&dst)[Lay::kKSteps][2], int r, int h) {
+        const uint32_t *qrow = (const uint32_t *)(p.q + ((size_t)r * p.num_q_heads + h * G + g_row) * D);
+#pragma unroll
+        for (int ks = 0; ks < Lay::kKSteps; ++ks) {
+            dst[ks][0] = g_row < G ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
+            dst[ks][1] = g_row < G ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
+        }
+    };
+
+    // Issue the loads of the tile under the issue cursor into stage issued % NS, then advance.
+    auto issue_next = [&]() {
+        const int ck = ic.tile / kTilesPerChunk;
+        if (ck != cur_chunk) {
+            cur_chunk = ck;
+            cur_val = nxt_val;
+            nxt_val = load_chunk(ic.r, ck + 1);
+        }
+        const int n_pages = (ic.L + kPageSize - 1) / kPageSize;
+        const int np = min(kPagesPerTile, n_pages - ic.tile * kPagesPerTile);
+        const int pg = lane / Lay::kHalves, hf = lane % Lay::kHalves;
+        int page = __shfl_sync(0xffffffffu, cur_val, ((ic.tile % kTilesPerChunk) * kPagesPerTile + pg) & 31);
+        const int slot = issued % NS;
+        fence_proxy_async();                      // this warp's earlier reads of the stage precede the copy
+        __syncwarp();
+        if (lane == 0) mbar_arrive_expect_tx(bars + slot * 8, np * Lay::kPageBytes);
+        __syncwarp();
+        if (lane < np * Lay::kHalves) {
+            if (page < 0 || page >= p.num_pages) {
+                atomicOr(p.status, kStatusBadPage);
+                page = 0;
+            }
+            const int y = ((p.layer_page_base + page) * p.num_kv_heads + ic.h) * 32;
+            tma_load_2d(ring + slot * Lay::kStageBytes + pg * Lay::kPageBytes + hf * Lay::kHalfBytes,
+                        &tmap, hf * 64, y, bars + slot * 8);
+        }
+        ++issued;
+        if (issued < n_total) {
+            ic.next(p);
+            if (ic.tile == 0) {
+                // entered a new (request, kv head): its first table chunk was fetched ahead
+                cur_chunk = 0;
+                cur_val = (pf_row == ic.r) ? pf_val : load_chunk(ic.r, 0);
+                nxt_val = load_chunk(ic.r, 1);
+                pf_row = (ic.h + 1 < p.num_kv_heads) ? ic.r : ic.r + 1;
+                pf_val = (pf_row == ic.r) ? cur_val : load_chunk(pf_row, 0);
+                if (qn_r < 0) {
+                    load_q(qn, ic.r, ic.h);
+                    qn_r = ic.r; qn_h = ic.h;
+                }
+            }
+        }
+    };
+
+    for (int k = 0; k < NS && k < n_total; ++k) issue_next();
+
+    // ---- compute side
+    SpanCursor cc;
+    cc.r = st.r; cc.h = st.h; cc.tile = st.tile; cc.L = st.L; cc.tiles = st.tiles_r;
+    const int g0 = (lane & 3) * 2;               // first of the two group columns this lane accumulates
+    uint32_t k_off[4], v_off[4];                 // ldmatrix lane offsets inside one page block
     {
         const int krow = (lane & 7) + ((lane >> 3) & 1) * 8;          // key row for matrices 0..3
         const int ksel = lane >> 4;                                    // second 16-byte chunk of the k16 step
@@ -503,43 +512,42 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         }
     }
 
-    int it = 0;
-    bool alive = true;
+    int done = 0;                                // tiles computed (or skipped after a wait gave up)
+    int landed = 0;                              // tiles whose copies were seen to complete
+    long long t_global = st.begin;               // global index of the compute cursor's tile
     bool first_piece = true;
-    while (wk.remaining > 0) {
-        const int n = wk.piece_tiles();
-        const bool complete = (wk.tile == 0 && n == wk.tiles);
+    while (done < n_total) {
+        const int n = min(cc.tiles - cc.tile, n_total - done);
+        const bool complete = (cc.tile == 0 && n == cc.tiles);
+        const int piece_r = cc.r, piece_h = cc.h, piece_L = cc.L, piece_tile0 = cc.tile, piece_tiles = cc.tiles;
 
-        // Q^T fragments of this (request, kv head): b0/b1 of k-step ks hold
-        // Q[g_row][ks*16 + 2*(lane%4) + {0,1}] and the same columns + 8.
         uint32_t qf[Lay::kKSteps][2];
-        {
-            const uint32_t *qrow = (const uint32_t *)(p.q + ((size_t)wk.r * p.num_q_heads + wk.h * G + g_row) * D);
+        if (qn_r == piece_r && qn_h == piece_h) {
 #pragma unroll
-            for (int ks = 0; ks < Lay::kKSteps; ++ks) {
-                qf[ks][0] = g_row < G ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
-                qf[ks][1] = g_row < G ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
-            }
+            for (int ks = 0; ks < Lay::kKSteps; ++ks) { qf[ks][0] = qn[ks][0]; qf[ks][1] = qn[ks][1]; }
+            qn_r = -1;
+        } else {
+            load_q(qf, piece_r, piece_h);
         }
         float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
         float o[Lay::kDTiles][4];
 #pragma unroll
         for (int dt = 0; dt < Lay::kDTiles; ++dt) o[dt][0] = o[dt][1] = o[dt][2] = o[dt][3] = 0.f;
 
-        for (int ti = wk.tile; ti < wk.tile + n; ++ti, ++it) {
-            if (it % W != warp) continue;
-            const int slot = it % S;
+        for (int ti = piece_tile0; ti < piece_tile0 + n; ++ti, ++done) {
+            const int slot = done % NS;
             if (alive) {
-                alive = mbar_wait_bounded(full_bar + slot * 8, (it / S) & 1, abort_flag, p.status);
+                alive = mbar_wait_bounded(bars + slot * 8, (done / NS) & 1, p.status);
                 alive = __all_sync(0xffffffffu, alive);
             }
             if (!alive) continue;
-            if (it == 0 && lane == 0) p.cta_trace[blockIdx.x * 4 + 1] = global_timer_ns();
+            ++landed;
+            if (done == 0 && lane == 0) p.trace[span * 4 + 1] = global_timer_ns();
 
-            const int ntok = min(kTileTokens, wk.L - ti * kTileTokens);     // valid tokens in this tile
+            const int ntok = min(kTileTokens, piece_L - ti * kTileTokens);      // valid tokens in this tile
             const bool full_tile = (ntok == kTileTokens);
             const int np = (ntok + kPageSize - 1) / kPageSize;
-            const uint32_t sb = stage_base + slot * Lay::kStageBytes;
+            const uint32_t sb = ring + slot * Lay::kStageBytes;
 
             if (!full_tile && (ntok & (kPageSize - 1))) {
                 // Value rows past the context's end hold whatever the pool holds; their weights are
@@ -553,7 +561,6 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                                        (16 + row0 + rem / 8) * 128 + (rem % 8) * 16;
                     asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
                 }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
             }
 
@@ -622,140 +629,120 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     }
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_bar + slot * 8);
+            // the stage is free again: refill it with the tile NS ahead
+            if (issued < n_total) issue_next();
         }
+        if (lane == 0 && done == n_total) p.trace[span * 4 + 2] = global_timer_ns();
 
-        // ---- merge the W warps' states of this piece and write it out
+        // ---- finish the piece: row sums across the warp, then through the staging tile
 #pragma unroll
         for (int x = 4; x < 32; x <<= 1) {
             l0 += __shfl_xor_sync(0xffffffffu, l0, x);
             l1 += __shfl_xor_sync(0xffffffffu, l1, x);
         }
-        {
-            float *so = scratch_o + (size_t)warp * D * kMaxGroup;
 #pragma unroll
-            for (int dt = 0; dt < Lay::kDTiles; ++dt) {
-                const int d = dt * 16 + (lane >> 2);
-                *(float2 *)(so + d * kMaxGroup + g0) = make_float2(o[dt][0], o[dt][1]);
-                *(float2 *)(so + (d + 8) * kMaxGroup + g0) = make_float2(o[dt][2], o[dt][3]);
+        for (int dt = 0; dt < Lay::kDTiles; ++dt) {
+            const int d = dt * 16 + (lane >> 2);
+            staging[g0 * Lay::kStagePitch + d] = o[dt][0];
+            staging[(g0 + 1) * Lay::kStagePitch + d] = o[dt][1];
+            staging[g0 * Lay::kStagePitch + d + 8] = o[dt][2];
+            staging[(g0 + 1) * Lay::kStagePitch + d + 8] = o[dt][3];
+        }
+        __syncwarp();
+        uint16_t *out_rows = p.out + ((size_t)piece_r * p.num_q_heads + piece_h * G) * D;
+        if (complete) {
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g) {
+                const float lg = __shfl_sync(0xffffffffu, (g & 1) ? l1 : l0, g >> 1);
+                if (g < G && lane * 4 < D) {
+                    const float4 a = *(const float4 *)(staging + g * Lay::kStagePitch + lane * 4);
+                    const float inv = 1.f / lg;
+                    uint2 packed;
+                    packed.x = pack_bf16x2(a.x * inv, a.y * inv);
+                    packed.y = pack_bf16x2(a.z * inv, a.w * inv);
+                    *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
+                }
             }
+        } else {
+            const int slot_id = 2 * span + (first_piece ? 0 : 1);
+            float *pa = p.part_acc + (size_t)slot_id * kMaxGroup * D;
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g)
+                if (lane * 4 < D)
+                    *(float4 *)(pa + g * D + lane * 4) = *(const float4 *)(staging + g * Lay::kStagePitch + lane * 4);
             if (lane < 4) {
-                float *ml = scratch_ml + warp * 2 * kMaxGroup;
+                float *ml = p.part_ml + slot_id * 2 * kMaxGroup;
                 ml[g0] = m0; ml[g0 + 1] = m1;
                 ml[kMaxGroup + g0] = l0; ml[kMaxGroup + g0 + 1] = l1;
             }
+            // ---- arrive; the last arriver of this (request, kv head) merges its partials
+            const long long item_begin = t_global - piece_tile0;
+            const long long item_end = item_begin + piece_tiles;
+            const int s_first = (int)(item_begin / q_span), s_last = (int)((item_end - 1) / q_span);
+            __threadfence();
+            __syncwarp();
+            int prior = 0;
+            if (lane == 0) prior = atomicAdd(p.arrivals + s_first, 1);
+            prior = __shfl_sync(0xffffffffu, prior, 0);
+            if (prior == s_last - s_first) {
+                __threadfence();
+                if (lane == 0) p.arrivals[s_first] = 0;          // ready for the next launch
+                const int pieces = s_last - s_first + 1;
+                const int slot_first = (item_begin == (long long)s_first * q_span) ? 2 * s_first : 2 * s_first + 1;
+                auto slot_of = [&](int i) { return i == 0 ? slot_first : 2 * (s_first + i); };
+                for (int g = 0; g < G; ++g) {
+                    float mstar = -INFINITY;
+                    for (int i = lane; i < pieces; i += 32)
+                        mstar = fmaxf(mstar, ld_cg_f32(p.part_ml + slot_of(i) * 2 * kMaxGroup + g));
+#pragma unroll
+                    for (int x = 16; x > 0; x >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, x));
+                    float lsum = 0.f;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int base = 0; base < pieces; base += 32) {
+                        // lane i of this round owns piece base + i: its factor and its share of the row sum
+                        float f_mine = 0.f;
+                        if (base + lane < pieces) {
+                            const float *ml = p.part_ml + slot_of(base + lane) * 2 * kMaxGroup;
+                            f_mine = fast_exp2(ld_cg_f32(ml + g) - mstar);
+                            lsum += f_mine * ld_cg_f32(ml + kMaxGroup + g);
+                        }
+                        const int cnt = min(32, pieces - base);
+#pragma unroll 4
+                        for (int i = 0; i < cnt; ++i) {
+                            const float f = __shfl_sync(0xffffffffu, f_mine, i);
+                            if (lane * 4 < D) {
+                                const float4 a = ld_cg_f32x4(p.part_acc + ((size_t)slot_of(base + i) * kMaxGroup + g) * D + lane * 4);
+                                acc.x += f * a.x; acc.y += f * a.y; acc.z += f * a.z; acc.w += f * a.w;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int x = 16; x > 0; x >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, x);
+                    if (lane * 4 < D) {
+                        const float inv = 1.f / lsum;
+                        uint2 packed;
+                        packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+                        packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+                        *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
+                    }
+                }
+            }
         }
-        named_barrier_sync(1, W * 32);
-        {
-            float f[W][kMaxGroup], mstar[kMaxGroup], lsum[kMaxGroup];
-#pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g) {
-                float mm = -INFINITY;
-#pragma unroll
-                for (int w = 0; w < W; ++w) mm = fmaxf(mm, scratch_ml[w * 2 * kMaxGroup + g]);
-                mstar[g] = mm;
-                float ls = 0.f;
-#pragma unroll
-                for (int w = 0; w < W; ++w) {
-                    f[w][g] = fast_exp2(scratch_ml[w * 2 * kMaxGroup + g] - mm);   // idle warp: exp2(-inf) = 0
-                    ls += f[w][g] * scratch_ml[w * 2 * kMaxGroup + kMaxGroup + g];
-                }
-                lsum[g] = ls;
-            }
-            const int slot_id = 2 * blockIdx.x + (first_piece ? 0 : 1);
-            for (int d = threadIdx.x; d < D; d += W * 32) {
-                float acc[kMaxGroup];
-#pragma unroll
-                for (int g = 0; g < kMaxGroup; ++g) acc[g] = 0.f;
-#pragma unroll
-                for (int w = 0; w < W; ++w) {
-                    const float4 a = *(const float4 *)(scratch_o + ((size_t)w * D + d) * kMaxGroup);
-                    const float4 b = *(const float4 *)(scratch_o + ((size_t)w * D + d) * kMaxGroup + 4);
-                    acc[0] += f[w][0] * a.x; acc[1] += f[w][1] * a.y; acc[2] += f[w][2] * a.z; acc[3] += f[w][3] * a.w;
-                    acc[4] += f[w][4] * b.x; acc[5] += f[w][5] * b.y; acc[6] += f[w][6] * b.z; acc[7] += f[w][7] * b.w;
-                }
-                if (complete) {
-#pragma unroll
-                    for (int g = 0; g < kMaxGroup; ++g)
-                        if (g < G)
-                            p.out[((size_t)wk.r * p.num_q_heads + wk.h * G + g) * D + d] = f32_to_bf16_rn(acc[g] / lsum[g]);
-                } else {
-#pragma unroll
-                    for (int g = 0; g < kMaxGroup; ++g)
-                        p.part_acc[((size_t)slot_id * kMaxGroup + g) * D + d] = acc[g];
-                }
-            }
-            if (!complete && threadIdx.x < kMaxGroup) {
-                p.part_ml[slot_id * 2 * kMaxGroup + threadIdx.x] = mstar[threadIdx.x];
-                p.part_ml[slot_id * 2 * kMaxGroup + kMaxGroup + threadIdx.x] = lsum[threadIdx.x];
-            }
-        }
-        named_barrier_sync(1, W * 32);            // scratch is reused by the next piece
+        __syncwarp();                             // staging is reused by the next piece
         first_piece = false;
-        wk.advance(p, n);
-    }
-    if (threadIdx.x == 0) p.cta_trace[blockIdx.x * 4 + 3] = global_timer_ns();
-}
-
-// ------------------------------------------------------------------------------------------
-// K4: log-sum-exp combine.  Block c looks at the boundary between spans c and c+1.  If that
-// boundary cuts a (request, kv head) and is the first one to cut it, the block merges all the
-// partials of that (request, kv head) and writes its bf16 output rows.
-// ------------------------------------------------------------------------------------------
-struct CombineParams {
-    const PlanHeader *header;
-    const int32_t *tile_prefix;
-    const float *part_acc;
-    const float *part_ml;
-    uint16_t *out;
-    int32_t batch, num_kv_heads, num_q_heads, group, head_dim;
-};
-
-__global__ void lse_combine_kernel(const CombineParams p)
-{
-    const int total = p.header->total_tiles;
-    const int q = p.header->tiles_per_cta;
-    const int c = blockIdx.x;
-    const long long tb = (long long)(c + 1) * q;            // first tile of span c + 1
-    if (tb >= total) return;
-
-    // (request, kv head) containing tile tb
-    int lo = 0, hi = p.batch;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if ((long long)p.tile_prefix[mid] * p.num_kv_heads > tb) hi = mid; else lo = mid;
-    }
-    const int r = lo;
-    const int tr = p.tile_prefix[r + 1] - p.tile_prefix[r];
-    const int rem = (int)(tb - (long long)p.tile_prefix[r] * p.num_kv_heads);
-    const int h = rem / tr, tile = rem % tr;
-    if (tile == 0) return;                                  // boundary falls between two pieces
-    const long long item_begin = tb - tile, item_end = item_begin + tr;
-    if ((long long)c * q > item_begin) return;              // an earlier boundary already cuts it
-
-    const int first_slot = ((long long)c * q == item_begin) ? 2 * c : 2 * c + 1;
-    int last_cta = c + 1;
-    while ((long long)(last_cta + 1) * q < item_end) ++last_cta;
-    const int pieces = last_cta - c + 1;
-
-    const int D = p.head_dim, G = p.group;
-    for (int idx = threadIdx.x; idx < G * D; idx += blockDim.x) {
-        const int g = idx / D, d = idx % D;
-        float mstar = -INFINITY;
-        for (int i = 0; i < pieces; ++i) {
-            const int slot = (i == 0) ? first_slot : 2 * (c + i);
-            mstar = fmaxf(mstar, p.part_ml[slot * 2 * kMaxGroup + g]);
+        t_global += n;
+        if (done < n_total) {
+            // move the compute cursor to the start of the next (request, kv head)
+            cc.tile = cc.tiles - 1;
+            cc.next(p);
         }
-        float lsum = 0.f, acc = 0.f;
-        for (int i = 0; i < pieces; ++i) {
-            const int slot = (i == 0) ? first_slot : 2 * (c + i);
-            const float f = fast_exp2(p.part_ml[slot * 2 * kMaxGroup + g] - mstar);
-            lsum += f * p.part_ml[slot * 2 * kMaxGroup + kMaxGroup + g];
-            acc += f * p.part_acc[((size_t)slot * kMaxGroup + g) * D + d];
-        }
-        p.out[((size_t)r * p.num_q_heads + h * G + g) * D + d] = f32_to_bf16_rn(acc / lsum);
     }
+
+    // Do not leave while copies into this warp's ring may still be in flight (only after a wait gave up).
+    if (!alive) {
+        for (int k = landed; k < issued; ++k) mbar_wait_bounded(bars + (k % NS) * 8, (k / NS) & 1, p.status);
+    }
+    if (lane == 0) p.trace[span * 4 + 3] = global_timer_ns();
 }
 
 }  // namespace ckv

@@ -59,7 +59,7 @@ def test_tiny_workload_append_bit_exact_and_attention_within_tolerance():
     assert_close(dev_to_bits(ds.out[0]), ref_out, "tiny")
 
 
-@pytest.mark.parametrize("partition", [1, 2, 3, 5, 31, 37, 148, 296, 1024])
+@pytest.mark.parametrize("partition", [1, 2, 3, 5, 31, 37, 148, 592, 1021, 2048])
 def test_partition_invariance_on_tiny_workload(partition):
     h = wl.host_inputs(wl.workload("tiny"))
     _, ref_out = oracle_step(h)
@@ -213,25 +213,31 @@ def test_too_long_length_and_bad_page_id_are_reported_without_faulting():
 
 # --------------------------------------------------------------------------- the plan
 
-def check_plan(kp, lens_np, Hkv):
-    sl = torch.from_numpy(lens_np).cuda()
-    hdr, starts = kp.decode_plan(sl)
-    tiles = (lens_np.astype(np.int64) + 63) // 64
+def expected_plan(lens_np, Hkv, C):
+    tiles = (lens_np.astype(np.int64) + 31) // 32
     prefix = np.concatenate([[0], np.cumsum(tiles)]) * Hkv
     total = int(prefix[-1])
-    C = kp.get_partition()
-    assert hdr["total_tiles"] == total and hdr["num_ctas"] == C
-    q = hdr["tiles_per_cta"]
-    assert q == max(1, -(-total // C))
-    assert hdr["ctas_with_work"] == -(-total // q)
+    q = max(1, -(-total // C))
+    starts = np.full((C, 4), -1, dtype=np.int32)
     for c in range(C):
         t0 = c * q
         if t0 >= total:
-            assert (starts[c] == -1).all()
             continue
         r = int(np.searchsorted(prefix, t0, side="right") - 1)
         rem = t0 - int(prefix[r])
-        assert starts[c].tolist() == [r, rem // int(tiles[r]), rem % int(tiles[r]), t0]
+        starts[c] = [r, rem // int(tiles[r]), rem % int(tiles[r]), t0]
+    return total, q, starts
+
+
+def check_plan(kp, lens_np, Hkv):
+    sl = torch.from_numpy(lens_np).cuda()
+    hdr, starts = kp.decode_plan(sl)
+    C = kp.get_partition()
+    total, q, want = expected_plan(lens_np, Hkv, C)
+    assert hdr["total_tiles"] == total and hdr["num_spans"] == C
+    assert hdr["tiles_per_span"] == q
+    assert hdr["spans_with_work"] == -(-total // q)
+    assert np.array_equal(starts, want)
     return hdr
 
 
@@ -242,12 +248,26 @@ def test_plan_partitions_tiles_evenly_and_deterministically():
         lens = wl.seq_lens(w)
         cfg = b.make_config(1, w.num_q_heads, w.num_kv_heads, w.head_dim, 64, int(wl.pages_of(lens).max()), lens.size)
         kp = b.KvPool(cfg)
-        for C in (kp.get_partition(), 1, 7, 296, 1024):
+        for C in (kp.get_partition(), 1, 7, 296, 2048):
             kp.set_partition(C)
             hdr = check_plan(kp, lens, w.num_kv_heads)
             hdr2, _ = kp.decode_plan(torch.from_numpy(lens).cuda())
             assert hdr == hdr2
         kp.close()
+
+
+def test_attention_kernel_derives_the_same_partition_as_the_plan():
+    h = custom_inputs([700, 90, 2000, 64, 1500, 333, 800, 16, 5000], 8, 2, 128, seed=71)
+    ds = make_device_step(h)
+    for C in (ds.pool.get_partition(), 5, 77):
+        ds.pool.set_partition(C)
+        ds.pool.decode_attention(0, ds.bt, ds.sl, ds.q[0], ds.out[0])
+        trace, starts = ds.pool.read_span_trace()
+        _, _, want = expected_plan(h.seq_lens, 2, C)
+        assert np.array_equal(starts, want)
+        busy = want[:, 0] >= 0
+        assert np.all(trace[busy, 3] >= trace[busy, 0]) and np.all(trace[busy, 1] > 0)
+    assert ds.pool.check_status() == 0
 
 
 # --------------------------------------------------------------------------- configs 2, 5
@@ -293,11 +313,11 @@ def full_parity(name, partitions=(None,)):
 
 
 def test_llama8b_batch64_full_parity():
-    full_parity("llama8b_b64", partitions=(None, 296, 100))
+    full_parity("llama8b_b64", partitions=(None, 296, 100, 2048))
 
 
 def test_skewed_long_context_full_parity():
-    full_parity("skewed_long", partitions=(None, 37))
+    full_parity("skewed_long", partitions=(None, 37, 2048))
 
 
 # --------------------------------------------------------------------------- host-buffer entry and sweep
@@ -324,7 +344,7 @@ def test_step_latency_sweep_runs_nested_prefixes_and_counts_launches():
     med, mn = ds.pool.step_latency_sweep([1, 2, 4, 8], ds.bt, ds.sl, ds.q, ds.k_new, ds.v_new, ds.out,
                                          warmup=2, iters=5)
     assert med.shape == (4,) and np.all(med > 0) and np.all(mn > 0) and np.all(mn <= med)
-    assert ds.pool.launch_count() - n0 == 4 * (2 + 5) * 2 * 4    # sizes * steps * layers * kernels
+    assert ds.pool.launch_count() - n0 == 4 * (2 + 5) * 2 * 2    # sizes * steps * layers * kernels
     # the last sweep point ran the full batch on both layers: outputs must be the oracle's
     sh = pool_shape(h.w, h.num_pages)
     ref_pool = h.pool.copy().reshape(-1)
@@ -357,7 +377,7 @@ def test_arguments_are_validated_on_the_host():
     with pytest.raises(b.CkvError):
         ds.pool.set_partition(0)
     with pytest.raises(b.CkvError):
-        ds.pool.set_partition(2000)
+        ds.pool.set_partition(3000)
     big = torch.zeros(9, dtype=torch.int32, device="cuda")
     with pytest.raises(b.CkvError):
         ds.pool.decode_attention(0, ds.bt, big, ds.q[0], ds.out[0])          # batch > max_batch

@@ -138,6 +138,16 @@ int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, vo
 int32_t ckv_set_partition(ckv_pool *pool, int32_t num_spans);
 int32_t ckv_get_partition(const ckv_pool *pool);
 
+/* Kernel overlap (default on): append and attention kernels are launched so that a kernel's
+ * prologue may run under the tail of its predecessor in the stream; each waits for the
+ * predecessor to complete before it first touches the pool, the workspace, q or an output.
+ * The attention prologue reads d_seq_lens and d_block_tables BEFORE that wait, so with overlap on
+ * they must not be produced by the kernel that immediately precedes decode_attention in the
+ * stream (tables copied by a memcpy, or written by any earlier kernel, are fine -- the usual case,
+ * since a serving engine uploads them once per iteration).  Turning overlap off restores plain
+ * stream order.  Errors: CKV_EINVAL. */
+int32_t ckv_set_overlap(ckv_pool *pool, int32_t enable);
+
 /* Synchronise `stream`, read and clear the device status word.  Returns CKV_OK, CKV_EBOUNDS
  * (bad length or page id seen), CKV_ETIMEOUT, or CKV_ECUDA.  *out_bits (may be NULL) receives
  * the raw CKV_STATUS_* bits. */

@@ -23,7 +23,7 @@ EXPORTS = (
     "kv_pool_bytes", "kv_workspace_bytes", "kv_pool_create", "kv_pool_destroy", "kv_append",
     "decode_attention", "decode_plan", "ckv_set_partition", "ckv_get_partition", "kv_check_status",
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
-    "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace",
+    "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace", "ckv_set_overlap",
 )
 
 
@@ -56,6 +56,7 @@ def _load() -> ctypes.CDLL:
     lib.decode_attention.restype = i32; lib.decode_attention.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.decode_plan.restype = i32; lib.decode_plan.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_set_partition.restype = i32; lib.ckv_set_partition.argtypes = [vp, i32]
+    lib.ckv_set_overlap.restype = i32; lib.ckv_set_overlap.argtypes = [vp, i32]
     lib.ckv_get_partition.restype = i32; lib.ckv_get_partition.argtypes = [vp]
     lib.kv_check_status.restype = i32; lib.kv_check_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.decode_step_host.restype = i32; lib.decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
@@ -178,6 +179,9 @@ class KvPool:
 
     def set_partition(self, num_spans: int) -> None:
         _check(lib.ckv_set_partition(self._h, int(num_spans)))
+
+    def set_overlap(self, enable: bool) -> None:
+        _check(lib.ckv_set_overlap(self._h, 1 if enable else 0))
 
     def get_partition(self) -> int:
         return int(lib.ckv_get_partition(self._h))

@@ -112,6 +112,7 @@ struct ckv_pool {
     CUtensorMap tmap;
     int64_t launches;
     bool profile;
+    bool overlap;                    // launch kernels with programmatic stream serialization
     std::vector<cudaEvent_t> ev;     // pairs (start, stop)
     int ev_used;
 
@@ -131,8 +132,17 @@ int32_t launch_attention(ckv_pool *pool, const ckv::AttnParams &ap, cudaStream_t
         configured_device = pool->device;
     }
     const int ctas = (pool->num_spans + W - 1) / W;
-    kernel<<<ctas, Lay::kThreads, Lay::kSmemBytes, stream>>>(pool->tmap, ap);
-    CKV_CUDA(cudaGetLastError());
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(ctas);
+    lc.blockDim = dim3(Lay::kThreads);
+    lc.dynamicSmemBytes = Lay::kSmemBytes;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pool->overlap ? 1 : 0;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    CKV_CUDA(cudaLaunchKernelEx(&lc, kernel, pool->tmap, ap));
     return CKV_OK;
 }
 
@@ -217,6 +227,7 @@ int32_t kv_pool_create(const ckv_config *cfg, void *d_pool, size_t pool_bytes, v
     p->ws = ws;
     p->launches = 0;
     p->profile = false;
+    p->overlap = true;
     p->ev_used = 0;
 
     // Tensor map over the whole pool seen as rows of head_dim bf16; one box = 32 rows (the 16 key
@@ -271,6 +282,13 @@ int32_t ckv_set_partition(ckv_pool *pool, int32_t num_spans)
 
 int32_t ckv_get_partition(const ckv_pool *pool) { return pool ? pool->num_spans : CKV_EINVAL; }
 
+int32_t ckv_set_overlap(ckv_pool *pool, int32_t enable)
+{
+    if (!pool) return fail(CKV_EINVAL, "ckv_set_overlap: pool is NULL");
+    pool->overlap = enable != 0;
+    return CKV_OK;
+}
+
 int64_t ckv_launch_count(const ckv_pool *pool) { return pool ? pool->launches : 0; }
 
 int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
@@ -296,8 +314,16 @@ int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d
     const long long work = (long long)batch * c.num_kv_heads * 2 * (c.head_dim / 8);
     const int threads = 256;
     const int blocks = (int)std::min<long long>((work + threads - 1) / threads, 4096);
-    ckv::kv_append_kernel<<<blocks, threads, 0, static_cast<cudaStream_t>(stream)>>>(ap);
-    CKV_CUDA(cudaGetLastError());
+    cudaLaunchConfig_t lc{};
+    lc.gridDim = dim3(blocks);
+    lc.blockDim = dim3(threads);
+    lc.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = pool->overlap ? 1 : 0;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    CKV_CUDA(cudaLaunchKernelEx(&lc, ckv::kv_append_kernel, ap));
     pool->launches += 1;
     return CKV_OK;
 }

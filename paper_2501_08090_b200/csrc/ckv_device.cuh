@@ -55,6 +55,10 @@ struct AppendParams {
 
 __global__ void kv_append_kernel(const AppendParams p)
 {
+    // The pool may still be read by the attention kernel launched before this one: let the next
+    // kernel start its prologue, then wait for the predecessor before the first write.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int vec_per_row = p.head_dim / 8;                       // 16-byte pieces per row
     const int per_req = p.num_kv_heads * 2 * vec_per_row;
     const long long total = (long long)p.batch * per_req;
@@ -101,24 +105,37 @@ struct SpanStart {
     int total, q;          // header values
 };
 
+// Requests with an unusable length get their output rows cleared and the status word flagged.
+// Executed by one warp of the grid.
+__device__ __forceinline__ void flag_unusable_requests(const int32_t *__restrict__ seq_lens, int batch,
+                                                       int max_pages_per_req, int lane, uint16_t *out,
+                                                       int out_row_elems, uint32_t *status)
+{
+    for (int base = 0; base < batch; base += 32) {
+        const int r = base + lane;
+        const bool bad = r < batch && tiles_of_length(__ldg(seq_lens + r), max_pages_per_req) == 0;
+        unsigned todo = __ballot_sync(0xffffffffu, bad);
+        if (todo && lane == 0) atomicOr(status, kStatusBadLength);
+        while (todo) {                                   // the whole warp clears one row at a time
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            uint16_t *row = out + (size_t)(base + src) * out_row_elems;
+            for (int i = lane; i < out_row_elems; i += 32) row[i] = 0;
+        }
+    }
+}
+
 // Executed by one whole warp.  Two passes over seq_lens: the total, then the request that holds
-// tile span*q.  If `zero_rows` is set (one warp of the grid), requests with an unusable length
-// get their output rows cleared and the status word flagged.
+// tile span*q.
 __device__ __forceinline__ SpanStart warp_plan(const int32_t *__restrict__ seq_lens, int batch, int max_pages_per_req,
-                                               int num_kv_heads, int num_spans, int span, int lane,
-                                               uint16_t *zero_rows, int out_row_elems, uint32_t *status)
+                                               int num_kv_heads, int num_spans, int span, int lane)
 {
     SpanStart s;
     int sum = 0;
     for (int base = 0; base < batch; base += 32) {
         const int r = base + lane;
         if (r < batch) {
-            const int t = tiles_of_length(__ldg(seq_lens + r), max_pages_per_req);
-            sum += t;
-            if (t == 0 && zero_rows != nullptr) {
-                atomicOr(status, kStatusBadLength);
-                for (int i = 0; i < out_row_elems; ++i) zero_rows[(size_t)r * out_row_elems + i] = 0;
-            }
+            sum += tiles_of_length(__ldg(seq_lens + r), max_pages_per_req);
         }
     }
 #pragma unroll
@@ -171,8 +188,7 @@ __global__ void splitkv_plan_kernel(const PlanParams p)
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
     for (int span = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; span < p.num_spans; span += warps) {
-        const SpanStart s = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span,
-                                      lane, nullptr, 0, nullptr);
+        const SpanStart s = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane);
         if (lane == 0) {
             p.span_start[span] = s.r < 0 ? make_int4(-1, -1, -1, -1) : make_int4(s.r, s.h, s.tile, s.begin);
             if (span == 0) {
@@ -241,6 +257,19 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
+// start while its predecessor in the stream still runs.  grid_dependency_wait() blocks until the
+// predecessor has completed and its writes are visible; without the attribute it returns at once.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+__device__ __forceinline__ void grid_launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
 __device__ __forceinline__ void fence_proxy_async()
@@ -342,6 +371,84 @@ struct AttnParams {
     float scale_log2;               // log2(e) / sqrt(d)
 };
 
+// Merge the partials of one (request, kv head) that spans s_first..s_last hold, and write its bf16
+// output rows.  Run by one whole warp (the last one to arrive for that pair).  Loads are issued in
+// batches so the merge costs a few L2 round trips, not one per partial.
+template <int D>
+__device__ __noinline__ void combine_partials(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
+                                              uint16_t *out_rows, int s_first, int s_last, int slot_first, int G,
+                                              int lane)
+{
+    const int pieces = s_last - s_first + 1;
+    auto slot_of = [&](int i) { return i == 0 ? slot_first : 2 * (s_first + i); };
+
+    float mstar[kMaxGroup];
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) mstar[g] = -INFINITY;
+    for (int base = 0; base < pieces; base += 32) {
+        if (base + lane < pieces) {
+            const float *ml = part_ml + slot_of(base + lane) * 2 * kMaxGroup;
+            const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
+            mstar[0] = fmaxf(mstar[0], a.x); mstar[1] = fmaxf(mstar[1], a.y);
+            mstar[2] = fmaxf(mstar[2], a.z); mstar[3] = fmaxf(mstar[3], a.w);
+            mstar[4] = fmaxf(mstar[4], b.x); mstar[5] = fmaxf(mstar[5], b.y);
+            mstar[6] = fmaxf(mstar[6], b.z); mstar[7] = fmaxf(mstar[7], b.w);
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g)
+#pragma unroll
+        for (int x = 16; x > 0; x >>= 1) mstar[g] = fmaxf(mstar[g], __shfl_xor_sync(0xffffffffu, mstar[g], x));
+
+    float lsum[kMaxGroup];
+    float4 acc[kMaxGroup];
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) { lsum[g] = 0.f; acc[g] = make_float4(0.f, 0.f, 0.f, 0.f); }
+    for (int base = 0; base < pieces; base += 32) {
+        // lane i of this round owns piece base + i: its factors and its share of the row sums
+        float f_mine[kMaxGroup];
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g) f_mine[g] = 0.f;
+        if (base + lane < pieces) {
+            const float *ml = part_ml + slot_of(base + lane) * 2 * kMaxGroup;
+            const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
+            const float4 c = ld_cg_f32x4(ml + 8), d = ld_cg_f32x4(ml + 12);
+            const float mi[kMaxGroup] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+            const float li[kMaxGroup] = {c.x, c.y, c.z, c.w, d.x, d.y, d.z, d.w};
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g) {
+                f_mine[g] = fast_exp2(mi[g] - mstar[g]);
+                lsum[g] += f_mine[g] * li[g];
+            }
+        }
+        const int cnt = min(32, pieces - base);
+#pragma unroll 2
+        for (int i = 0; i < cnt; ++i) {
+            const float *pa = part_acc + (size_t)slot_of(base + i) * kMaxGroup * D + lane * 4;
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g) {
+                const float f = __shfl_sync(0xffffffffu, f_mine[g], i);
+                if (g < G && lane * 4 < D) {
+                    const float4 a = ld_cg_f32x4(pa + g * D);
+                    acc[g].x += f * a.x; acc[g].y += f * a.y; acc[g].z += f * a.z; acc[g].w += f * a.w;
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) {
+#pragma unroll
+        for (int x = 16; x > 0; x >>= 1) lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], x);
+        if (g < G && lane * 4 < D) {
+            const float inv = 1.f / lsum[g];
+            uint2 packed;
+            packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
+            packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
+            *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
+        }
+    }
+}
+
 template <int D, int W, int NS>
 struct AttnLayout {
     static constexpr int kHalves = D / 64;                       // 128-byte column blocks per row
@@ -392,6 +499,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     float *staging = (float *)(smem + Lay::kRingBytes + warp * Lay::kStagingBytes);
     const uint32_t bars = smem_u32(smem + Lay::kRingBytes + W * Lay::kStagingBytes) + warp * NS * 8;
 
+    grid_launch_dependents();
     if (span >= p.num_spans) return;
     unsigned long long t_start = 0;
     if (lane == 0) {
@@ -403,14 +511,19 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     __syncwarp();
 
     // ---- plan: where does this warp's span start?
-    const SpanStart st = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane,
-                                   span == 0 ? p.out : nullptr, p.num_q_heads * D, p.status);
-    if (lane == 0) {
-        p.span_start[span] = st.r < 0 ? make_int4(-1, -1, -1, -1) : make_int4(st.r, st.h, st.tile, st.begin);
-        p.trace[span * 4 + 0] = t_start;
-        p.trace[span * 4 + 1] = 0;
+    // Nothing read up to the dependency wait below is written by the preceding kernel of a decode
+    // step (the KV append writes only the pool), so this prologue overlaps that kernel's tail.
+    const SpanStart st = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane);
+    if (st.r < 0 || span == 0) {
+        grid_dependency_wait();
+        if (span == 0) flag_unusable_requests(p.seq_lens, p.batch, p.max_pages_per_req, lane, p.out, p.num_q_heads * D, p.status);
     }
     if (st.r < 0) {
+        if (lane == 0) {
+            p.span_start[span] = make_int4(-1, -1, -1, -1);
+            p.trace[span * 4 + 0] = t_start;
+            p.trace[span * 4 + 1] = 0;
+        }
         if (lane == 0) p.trace[span * 4 + 2] = p.trace[span * 4 + 3] = global_timer_ns();
         return;
     }
@@ -493,6 +606,12 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         }
     };
 
+    grid_dependency_wait();                       // the pool, the workspace and `out` are ours from here on
+    if (lane == 0) {
+        p.span_start[span] = make_int4(st.r, st.h, st.tile, st.begin);
+        p.trace[span * 4 + 0] = t_start;
+        p.trace[span * 4 + 1] = 0;
+    }
     for (int k = 0; k < NS && k < n_total; ++k) issue_next();
 
     // ---- compute side
@@ -516,6 +635,9 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     int landed = 0;                              // tiles whose copies were seen to complete
     long long t_global = st.begin;               // global index of the compute cursor's tile
     bool first_piece = true;
+    // a span writes at most two partials: its first piece and its last piece
+    int pend_first[2] = {-1, -1}, pend_last[2] = {0, 0}, pend_slot[2] = {0, 0};
+    uint16_t *pend_out[2] = {nullptr, nullptr};
     while (done < n_total) {
         const int n = min(cc.tiles - cc.tile, n_total - done);
         const bool complete = (cc.tile == 0 && n == cc.tiles);
@@ -675,58 +797,15 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 ml[g0] = m0; ml[g0 + 1] = m1;
                 ml[kMaxGroup + g0] = l0; ml[kMaxGroup + g0 + 1] = l1;
             }
-            // ---- arrive; the last arriver of this (request, kv head) merges its partials
+            // ---- remember the arrival; it is made once the whole span has been streamed, so that
+            // neither the fence nor a merge ever interrupts this warp's loads
             const long long item_begin = t_global - piece_tile0;
             const long long item_end = item_begin + piece_tiles;
-            const int s_first = (int)(item_begin / q_span), s_last = (int)((item_end - 1) / q_span);
-            __threadfence();
-            __syncwarp();
-            int prior = 0;
-            if (lane == 0) prior = atomicAdd(p.arrivals + s_first, 1);
-            prior = __shfl_sync(0xffffffffu, prior, 0);
-            if (prior == s_last - s_first) {
-                __threadfence();
-                if (lane == 0) p.arrivals[s_first] = 0;          // ready for the next launch
-                const int pieces = s_last - s_first + 1;
-                const int slot_first = (item_begin == (long long)s_first * q_span) ? 2 * s_first : 2 * s_first + 1;
-                auto slot_of = [&](int i) { return i == 0 ? slot_first : 2 * (s_first + i); };
-                for (int g = 0; g < G; ++g) {
-                    float mstar = -INFINITY;
-                    for (int i = lane; i < pieces; i += 32)
-                        mstar = fmaxf(mstar, ld_cg_f32(p.part_ml + slot_of(i) * 2 * kMaxGroup + g));
-#pragma unroll
-                    for (int x = 16; x > 0; x >>= 1) mstar = fmaxf(mstar, __shfl_xor_sync(0xffffffffu, mstar, x));
-                    float lsum = 0.f;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int base = 0; base < pieces; base += 32) {
-                        // lane i of this round owns piece base + i: its factor and its share of the row sum
-                        float f_mine = 0.f;
-                        if (base + lane < pieces) {
-                            const float *ml = p.part_ml + slot_of(base + lane) * 2 * kMaxGroup;
-                            f_mine = fast_exp2(ld_cg_f32(ml + g) - mstar);
-                            lsum += f_mine * ld_cg_f32(ml + kMaxGroup + g);
-                        }
-                        const int cnt = min(32, pieces - base);
-#pragma unroll 4
-                        for (int i = 0; i < cnt; ++i) {
-                            const float f = __shfl_sync(0xffffffffu, f_mine, i);
-                            if (lane * 4 < D) {
-                                const float4 a = ld_cg_f32x4(p.part_acc + ((size_t)slot_of(base + i) * kMaxGroup + g) * D + lane * 4);
-                                acc.x += f * a.x; acc.y += f * a.y; acc.z += f * a.z; acc.w += f * a.w;
-                            }
-                        }
-                    }
-#pragma unroll
-                    for (int x = 16; x > 0; x >>= 1) lsum += __shfl_xor_sync(0xffffffffu, lsum, x);
-                    if (lane * 4 < D) {
-                        const float inv = 1.f / lsum;
-                        uint2 packed;
-                        packed.x = pack_bf16x2(acc.x * inv, acc.y * inv);
-                        packed.y = pack_bf16x2(acc.z * inv, acc.w * inv);
-                        *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
-                    }
-                }
-            }
+            const int k = first_piece ? 0 : 1;
+            pend_first[k] = (int)(item_begin / q_span);
+            pend_last[k] = (int)((item_end - 1) / q_span);
+            pend_slot[k] = (item_begin == (long long)pend_first[k] * q_span) ? 2 * pend_first[k] : 2 * pend_first[k] + 1;
+            pend_out[k] = out_rows;
         }
         __syncwarp();                             // staging is reused by the next piece
         first_piece = false;
@@ -735,6 +814,24 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             // move the compute cursor to the start of the next (request, kv head)
             cc.tile = cc.tiles - 1;
             cc.next(p);
+        }
+    }
+
+    // ---- arrivals: whichever warp arrives last for a (request, kv head) merges its partials (wait-free)
+    if (pend_first[0] >= 0 || pend_first[1] >= 0) {
+        __threadfence();
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            if (pend_first[k] < 0) continue;
+            int prior = 0;
+            if (lane == 0) prior = atomicAdd(p.arrivals + pend_first[k], 1);
+            prior = __shfl_sync(0xffffffffu, prior, 0);
+            if (prior == pend_last[k] - pend_first[k]) {
+                __threadfence();
+                if (lane == 0) p.arrivals[pend_first[k]] = 0;        // ready for the next launch
+                combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k], pend_slot[k], G, lane);
+            }
         }
     }
 

@@ -108,10 +108,7 @@ class DeviceWorkload:
     def __init__(self, name: str, device, seed_offset: int = 0, batch=None, num_layers=None):
         import torch
         from paper_2501_08090_b200 import binding
-        w = wl.workload(name) if num_layers is None else wl.workload(name, num_layers=num_layers)
-        if seed_offset:
-            w = wl.workload(name, seed=w.seed + 1000 * seed_offset,
-                            **({"num_layers": num_layers} if num_layers is not None else {}))
+        w = rank_workload(name, seed_offset, num_layers)
         self.w, self.device = w, device
         self.lens = wl.seq_lens(w, batch)
         self.B = int(self.lens.size)
@@ -153,6 +150,14 @@ class DeviceWorkload:
                     raise binding.CkvError(rc, binding.last_error())
 
 
+def rank_workload(name: str, rank: int = 0, num_layers=None) -> "wl.Workload":
+    """The workload of one serving instance: same shape on every rank, its own seeded batch."""
+    over = {} if num_layers is None else {"num_layers": num_layers}
+    if rank:
+        over["seed"] = wl.workload(name).seed + 1000 * rank
+    return wl.workload(name, **over)
+
+
 def dist_setup(n_gpus: int):
     """(rank, world, local_rank); initialises NCCL only when launched under torchrun."""
     import torch
@@ -168,14 +173,14 @@ def dist_setup(n_gpus: int):
     return rank, world, local
 
 
-def reduce_max_sum(t_ms: float, units: float, world: int):
+def reduce_max_sum(t_ms: float, units: float, world: int, device="cuda"):
     """Max over ranks of the time, sum over ranks of the units (bytes, launches ...)."""
     if world == 1:
         return t_ms, units
     import torch
     import torch.distributed as dist
-    a = torch.tensor([t_ms], dtype=torch.float64, device="cuda")
-    b = torch.tensor([units], dtype=torch.float64, device="cuda")
+    a = torch.tensor([t_ms], dtype=torch.float64, device=device)
+    b = torch.tensor([units], dtype=torch.float64, device=device)
     dist.all_reduce(a, op=dist.ReduceOp.MAX)
     dist.all_reduce(b, op=dist.ReduceOp.SUM)
     return float(a.item()), float(b.item())

@@ -204,6 +204,44 @@ int32_t ckv_read_span_trace(ckv_pool *pool, void *stream, uint64_t *h_trace, int
 /* Kernels launched through this handle since creation (append, attention, plan inspection). */
 int64_t ckv_launch_count(const ckv_pool *pool);
 
+/*
+ * decode_attention without a workspace.  (The paper has no counterpart; this entry point exists
+ * for integration reasons only.)
+ *
+ * Who it is for: code that must not, or cannot, allocate device memory at the point where it
+ * needs attention -- an engine that handed all free HBM to the KV pool at start-up so that any
+ * later cudaMalloc fails, a plugin running under a host framework that owns the allocator, a
+ * latency-critical loop that cannot afford cudaMalloc's implicit device-wide synchronisation.
+ * Such a caller has the pool, the tables and q/out, but nowhere to put the split-KV partials.
+ *
+ * Here they go into a fixed array inside the library's device image instead:
+ * about 5.1 MiB per GPU, held by every GPU that loads the library until the process exits.  It is
+ * sized for at most 640 spans (a B200 uses 592) at head_dim <= 128.  No pool handle is needed: the
+ * configuration and the pool pointer are passed directly, on the CURRENT device.  The function
+ * calls no cudaMalloc / cudaFree and no allocating library routine; the result is the same as
+ * decode_attention's for the same partition.
+ *
+ *   cfg        shape of the pool (same rules as kv_pool_create; max_batch bounds `batch`)
+ *   d_pool     256-byte aligned device pointer to kv_pool_bytes(cfg) bytes
+ *   num_spans  partition width; 0 = warps per CTA x number of SMs.  More than 640 is rejected
+ *              with CKV_EINVAL and a message -- nothing is launched.
+ *   h_status   NULL: the call only enqueues work on `stream`.  Otherwise the call synchronises
+ *              `stream`, stores the CKV_STATUS_* bits there and returns CKV_EBOUNDS /
+ *              CKV_ETIMEOUT if any is set.
+ *
+ * Set-up: the first call on each device looks up the array's device address
+ * (cudaGetSymbolAddress) and remembers it; make that first call outside any stream capture.
+ * Sharing: every call on a device uses the same array, which still holds the previous call's
+ * contents; each call clears the parts that must start at zero (status word, arrival counters) on
+ * `stream` before its kernel.  Two calls that can overlap on the GPU (different streams, no
+ * dependency) would race on the array: keep calls on one device ordered.
+ * Errors: CKV_EINVAL (shape, alignment, layer/batch range, num_spans > 640), CKV_ECUDA.
+ */
+int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int32_t layer, int32_t batch,
+                                 const int32_t *d_block_tables, const int32_t *d_seq_lens,
+                                 const void *d_q, void *d_out, int32_t num_spans, void *stream,
+                                 uint32_t *h_status);
+
 /* Message describing the calling thread's most recent failure ("" if none). */
 const char *ckv_last_error(void);
 

@@ -24,6 +24,7 @@ EXPORTS = (
     "decode_attention", "decode_plan", "ckv_set_partition", "ckv_get_partition", "kv_check_status",
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
     "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace", "ckv_set_overlap",
+    "decode_attention_noalloc",
 )
 
 
@@ -66,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.ckv_profile_read.restype = i32
     lib.ckv_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(i32)]
     lib.ckv_read_span_trace.restype = i32; lib.ckv_read_span_trace.argtypes = [vp, vp, vp, vp]
+    lib.decode_attention_noalloc.restype = i32
+    lib.decode_attention_noalloc.argtypes = [cfgp, vp, i32, i32, vp, vp, vp, vp, i32, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.ckv_launch_count.restype = i64; lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_last_error.restype = ctypes.c_char_p; lib.ckv_last_error.argtypes = []
     return lib
@@ -240,3 +243,17 @@ class KvPool:
 
     def launch_count(self) -> int:
         return int(lib.ckv_launch_count(self._h))
+
+
+def decode_attention_noalloc(cfg: Config, pool: torch.Tensor, layer: int, block_tables, seq_lens, q, out,
+                             num_spans: int = 0, stream=None, sync: bool = True) -> int:
+    """decode_attention for callers that cannot allocate a workspace: partial results go into a fixed
+    array inside the library (at most 640 spans).  Runs on the current CUDA device.  With `sync`
+    the stream is synchronised and the device status bits are returned (and raised if non-zero)."""
+    bits = ctypes.c_uint32(0)
+    rc = lib.decode_attention_noalloc(ctypes.byref(cfg), _dev_ptr(pool), int(layer), int(seq_lens.shape[0]),
+                                      _dev_ptr(block_tables, torch.int32), _dev_ptr(seq_lens, torch.int32),
+                                      _dev_ptr(q, torch.bfloat16), _dev_ptr(out, torch.bfloat16), int(num_spans),
+                                      _stream_ptr(stream), ctypes.byref(bits) if sync else None)
+    _check(rc)
+    return int(bits.value)

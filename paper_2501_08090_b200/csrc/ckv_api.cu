@@ -175,6 +175,39 @@ int32_t launch_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, cu
     return CKV_OK;
 }
 
+// ------------------------------------------------------------------------------------------
+// Scratch for decode_attention_noalloc: lives in the library image, one copy per GPU that loads
+// it, for the life of the process.  Sized for kNoAllocMaxSpans spans at head_dim 128.
+// ------------------------------------------------------------------------------------------
+constexpr int kNoAllocMaxSpans = 640;
+constexpr size_t kNaStatus = 0;                                                       // 256 B
+constexpr size_t kNaArrivals = 256;                                                   // int32 [640]
+constexpr size_t kNaSpanStart = kNaArrivals + sizeof(int32_t) * kNoAllocMaxSpans;     // int4 [640]
+constexpr size_t kNaTrace = kNaSpanStart + sizeof(int4) * kNoAllocMaxSpans;           // u64 [640][4]
+constexpr size_t kNaPartMl = kNaTrace + sizeof(unsigned long long) * 4 * kNoAllocMaxSpans;
+constexpr size_t kNaPartAcc = kNaPartMl + sizeof(float) * 2 * kNoAllocMaxSpans * 2 * ckv::kMaxGroup;
+constexpr size_t kNoAllocScratchBytes = kNaPartAcc + sizeof(float) * 2 * kNoAllocMaxSpans * ckv::kMaxGroup * 128;
+static_assert(kNaSpanStart % 16 == 0 && kNaTrace % 8 == 0 && kNaPartMl % 16 == 0 && kNaPartAcc % 256 == 0,
+              "sub-buffers of the static scratch must keep their natural alignment");
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+// Device address of g_noalloc_scratch on each device (0 = not looked up yet).  In host code the
+// symbol's name is only a handle; the address a kernel can use comes from cudaGetSymbolAddress.
+unsigned char *g_noalloc_ptr[kMaxDevices] = {};
+
+template <int D, int W, int NS>
+int32_t launch_attention_noalloc(const CUtensorMap &tmap, const ckv::AttnParams &ap, cudaStream_t stream)
+{
+    using Lay = ckv::AttnLayout<D, W, NS>;
+    auto kernel = ckv::paged_decode_attn_kernel<D, W, NS>;
+    CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
+    kernel<<<(ap.num_spans + W - 1) / W, Lay::kThreads, Lay::kSmemBytes, stream>>>(tmap, ap);
+    CKV_CUDA(cudaGetLastError());
+    return CKV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -532,6 +565,102 @@ int32_t ckv_profile_read(ckv_pool *pool, double *out_attention_ms, int32_t *out_
     }
     *out_attention_ms = total;
     *out_launches = pool->ev_used;
+    return CKV_OK;
+}
+
+int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int32_t layer, int32_t batch,
+                                 const int32_t *d_block_tables, const int32_t *d_seq_lens, const void *d_q,
+                                 void *d_out, int32_t num_spans, void *stream, uint32_t *h_status)
+{
+    const char *why;
+    if (!config_ok(cfg, &why)) return fail(CKV_EINVAL, "decode_attention_noalloc: %s", why);
+    if (!d_pool || !d_block_tables || !d_seq_lens || !d_q || !d_out)
+        return fail(CKV_EINVAL, "decode_attention_noalloc: NULL argument");
+    if (reinterpret_cast<uintptr_t>(d_pool) & 255u) return fail(CKV_EINVAL, "decode_attention_noalloc: d_pool not 256-byte aligned");
+    if (!aligned16(d_q) || !aligned16(d_out)) return fail(CKV_EINVAL, "decode_attention_noalloc: q/out not 16-byte aligned");
+    if (layer < 0 || layer >= cfg->num_layers) return fail(CKV_EINVAL, "decode_attention_noalloc: layer %d outside [0, %d)", layer, cfg->num_layers);
+    if (batch < 1 || batch > cfg->max_batch) return fail(CKV_EINVAL, "decode_attention_noalloc: batch %d outside [1, %d]", batch, cfg->max_batch);
+
+    int device = -1;
+    CKV_CUDA(cudaGetDevice(&device));
+    if (device < 0 || device >= kMaxDevices) return fail(CKV_EINVAL, "decode_attention_noalloc: device ordinal %d not supported", device);
+    int cc_major = 0, sms = 0;
+    CKV_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, device));
+    CKV_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    if (cc_major != 10) return fail(CKV_ECUDA, "decode_attention_noalloc: device %d is sm_%dx; this library is built for sm_100a only", device, cc_major);
+
+    const int warps = cfg->head_dim == 128 ? kWarps128 : kWarps64;
+    if (num_spans == 0) num_spans = sms * warps;
+    if (num_spans < 1 || num_spans > kNoAllocMaxSpans)
+        return fail(CKV_EINVAL, "decode_attention_noalloc: %d spans requested, the built-in scratch holds partial results "
+                                "for at most %d (use decode_attention with a caller-provided workspace for more)",
+                    num_spans, kNoAllocMaxSpans);
+
+    // One-time set-up per device: the device address of the static scratch.
+    if (g_noalloc_ptr[device] == nullptr) {
+        unsigned char *ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void **>(&ptr), g_noalloc_scratch);
+        if (e != cudaSuccess || ptr == nullptr)
+            return fail(CKV_ECUDA, "decode_attention_noalloc: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+        g_noalloc_ptr[device] = ptr;
+    }
+    unsigned char *scratch = g_noalloc_ptr[device];
+
+    // Tensor map over the caller's pool, built on the stack (a host-side encode, no allocation).
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t ee = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (ee != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+        return fail(CKV_ECUDA, "decode_attention_noalloc: cuTensorMapEncodeTiled not available (%s)", cudaGetErrorString(ee));
+    CUtensorMap tmap;
+    const cuuint64_t rows = (cuuint64_t)cfg->num_layers * cfg->num_pages * cfg->num_kv_heads * 32;
+    const cuuint64_t dims[2] = {(cuuint64_t)cfg->head_dim, rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cfg->head_dim * 2};
+    const cuuint32_t box[2] = {64, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult cr = reinterpret_cast<EncodeTiledFn>(fn)(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(d_pool),
+                                                      dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return fail(CKV_ECUDA, "decode_attention_noalloc: cuTensorMapEncodeTiled returned %d", (int)cr);
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // The scratch keeps whatever the previous call left: the status word and the arrival counters
+    // must start at zero (partials, span starts and the timeline are fully rewritten before use).
+    CKV_CUDA(cudaMemsetAsync(scratch + kNaStatus, 0, kNaSpanStart - kNaStatus, s));
+
+    ckv::AttnParams ap{};
+    ap.block_tables = d_block_tables;
+    ap.seq_lens = d_seq_lens;
+    ap.q = static_cast<const uint16_t *>(d_q);
+    ap.out = static_cast<uint16_t *>(d_out);
+    ap.part_acc = reinterpret_cast<float *>(scratch + kNaPartAcc);
+    ap.part_ml = reinterpret_cast<float *>(scratch + kNaPartMl);
+    ap.arrivals = reinterpret_cast<int32_t *>(scratch + kNaArrivals);
+    ap.span_start = reinterpret_cast<int4 *>(scratch + kNaSpanStart);
+    ap.trace = reinterpret_cast<unsigned long long *>(scratch + kNaTrace);
+    ap.status = reinterpret_cast<uint32_t *>(scratch + kNaStatus);
+    ap.batch = batch;
+    ap.max_pages_per_req = cfg->max_pages_per_req;
+    ap.num_pages = cfg->num_pages;
+    ap.num_kv_heads = cfg->num_kv_heads;
+    ap.num_q_heads = cfg->num_q_heads;
+    ap.group = cfg->num_q_heads / cfg->num_kv_heads;
+    ap.layer_page_base = layer * cfg->num_pages;
+    ap.num_spans = num_spans;
+    ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)cfg->head_dim));
+
+    int32_t rc;
+    if (cfg->head_dim == 128) rc = launch_attention_noalloc<128, kWarps128, kStages128>(tmap, ap, s);
+    else rc = launch_attention_noalloc<64, kWarps64, kStages64>(tmap, ap, s);
+    if (rc) return rc;
+
+    if (h_status) {
+        CKV_CUDA(cudaMemcpyAsync(h_status, scratch + kNaStatus, sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
+        CKV_CUDA(cudaStreamSynchronize(s));
+        if (*h_status & ckv::kStatusWaitLimit) return fail(CKV_ETIMEOUT, "device status 0x%x: a bounded wait gave up", *h_status);
+        if (*h_status) return fail(CKV_EBOUNDS, "device status 0x%x: context length or page id out of range", *h_status);
+    }
     return CKV_OK;
 }
 

@@ -194,8 +194,10 @@ int32_t ckv_profile_read(ckv_pool *pool, double *out_attention_ms, int32_t *out_
 
 /*
  * Per-span timeline of the most recent attention kernel, for load-balance analysis (synchronises
- * `stream`).  h_trace: uint64 [ckv_get_partition()][4], nanoseconds of the GPU's global timer:
- * warp start, first tile landed (0 if the span had no work), last tile computed, span finished.
+ * `stream`).  h_trace: uint64 [ckv_get_partition()][8]: nanoseconds of the GPU's global timer at
+ * warp start, first tile landed (0 if the span had no work), last tile computed, span finished;
+ * then nanoseconds spent waiting for tile data, nanoseconds spent between pieces, the span's tile
+ * count and its piece count.
  * h_span_start (may be NULL): int32 [ckv_get_partition()][4], the span starts the kernel derived
  * itself, in decode_plan's format.  Errors: CKV_EINVAL, CKV_ECUDA.
  */

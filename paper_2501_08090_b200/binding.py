@@ -234,9 +234,10 @@ class KvPool:
         return float(ms.value), int(n.value)
 
     def read_span_trace(self, stream=None):
-        """(uint64 [spans][4] ns: warp start, first tile landed, last tile computed, span finished;
+        """(uint64 [spans][8]: ns of warp start, first tile landed, last tile computed, span finished;
+        ns spent waiting for data, ns spent between pieces; tiles; pieces.
         int32 [spans][4] span starts as the attention kernel derived them)."""
-        trace = np.zeros((self.get_partition(), 4), dtype=np.uint64)
+        trace = np.zeros((self.get_partition(), 8), dtype=np.uint64)
         starts = np.zeros((self.get_partition(), 4), dtype=np.int32)
         _check(lib.ckv_read_span_trace(self._h, _stream_ptr(stream), trace.ctypes.data, starts.ctypes.data))
         return trace, starts

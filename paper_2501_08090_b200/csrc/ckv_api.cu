@@ -35,8 +35,20 @@ int32_t fail(int32_t code, const char *fmt, ...)
     } while (0)
 
 // Attention kernel shapes: warps per CTA (one CTA per SM) and ring stages per warp.
-constexpr int kWarps128 = 4, kStages128 = 3;     // head_dim 128: 4 warps x 3 stages x 16 KB = 192 KB per SM
-constexpr int kWarps64 = 4, kStages64 = 4;       // head_dim 64:  4 warps x 4 stages x 8 KB
+#ifndef CKV_WARPS128
+#define CKV_WARPS128 4
+#endif
+#ifndef CKV_STAGES128
+#define CKV_STAGES128 3
+#endif
+#ifndef CKV_WARPS64
+#define CKV_WARPS64 4
+#endif
+#ifndef CKV_STAGES64
+#define CKV_STAGES64 4
+#endif
+constexpr int kWarps128 = CKV_WARPS128, kStages128 = CKV_STAGES128;   // head_dim 128: 4 warps x 3 stages x 16 KB = 192 KB per SM
+constexpr int kWarps64 = CKV_WARPS64, kStages64 = CKV_STAGES64;       // head_dim 64:  4 warps x 4 stages x 8 KB
 constexpr int kMaxProfile = 4096;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -83,7 +95,7 @@ WorkspaceLayout carve(const ckv_config &c)
     w.part_acc = take(sizeof(float) * 2 * ckv::kMaxSpans * ckv::kMaxGroup * c.head_dim);
     w.part_ml = take(sizeof(float) * 2 * ckv::kMaxSpans * 2 * ckv::kMaxGroup);
     w.arrivals = take(sizeof(int32_t) * ckv::kMaxSpans);
-    w.trace = take(sizeof(unsigned long long) * 4 * ckv::kMaxSpans);
+    w.trace = take(sizeof(unsigned long long) * 8 * ckv::kMaxSpans);
     w.st_tables = take(sizeof(int32_t) * (size_t)c.max_batch * c.max_pages_per_req);
     w.st_lens = take(sizeof(int32_t) * (size_t)c.max_batch);
     w.st_q = take((size_t)c.max_batch * c.num_q_heads * d2);
@@ -183,8 +195,8 @@ constexpr int kNoAllocMaxSpans = 640;
 constexpr size_t kNaStatus = 0;                                                       // 256 B
 constexpr size_t kNaArrivals = 256;                                                   // int32 [640]
 constexpr size_t kNaSpanStart = kNaArrivals + sizeof(int32_t) * kNoAllocMaxSpans;     // int4 [640]
-constexpr size_t kNaTrace = kNaSpanStart + sizeof(int4) * kNoAllocMaxSpans;           // u64 [640][4]
-constexpr size_t kNaPartMl = kNaTrace + sizeof(unsigned long long) * 4 * kNoAllocMaxSpans;
+constexpr size_t kNaTrace = kNaSpanStart + sizeof(int4) * kNoAllocMaxSpans;           // u64 [640][8]
+constexpr size_t kNaPartMl = kNaTrace + sizeof(unsigned long long) * 8 * kNoAllocMaxSpans;
 constexpr size_t kNaPartAcc = kNaPartMl + sizeof(float) * 2 * kNoAllocMaxSpans * 2 * ckv::kMaxGroup;
 constexpr size_t kNoAllocScratchBytes = kNaPartAcc + sizeof(float) * 2 * kNoAllocMaxSpans * ckv::kMaxGroup * 128;
 static_assert(kNaSpanStart % 16 == 0 && kNaTrace % 8 == 0 && kNaPartMl % 16 == 0 && kNaPartAcc % 256 == 0,
@@ -535,7 +547,7 @@ int32_t ckv_read_span_trace(ckv_pool *pool, void *stream, uint64_t *h_trace, int
 {
     if (!pool || !h_trace) return fail(CKV_EINVAL, "ckv_read_span_trace: NULL argument");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    CKV_CUDA(cudaMemcpyAsync(h_trace, pool->d_ws + pool->ws.trace, sizeof(uint64_t) * 4 * pool->num_spans,
+    CKV_CUDA(cudaMemcpyAsync(h_trace, pool->d_ws + pool->ws.trace, sizeof(uint64_t) * 8 * pool->num_spans,
                              cudaMemcpyDeviceToHost, s));
     if (h_span_start)
         CKV_CUDA(cudaMemcpyAsync(h_span_start, pool->d_ws + pool->ws.span_start, sizeof(int4) * pool->num_spans,

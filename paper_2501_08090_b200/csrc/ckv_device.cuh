@@ -12,7 +12,10 @@
 namespace ckv {
 
 constexpr int kPageSize = 16;        // tokens per page
-constexpr int kPagesPerTile = 2;     // a tile is the scheduling unit: 32 tokens of one (request, kv head)
+#ifndef CKV_PAGES_PER_TILE
+#define CKV_PAGES_PER_TILE 2
+#endif
+constexpr int kPagesPerTile = CKV_PAGES_PER_TILE;   // a tile is the scheduling unit: 32 tokens of one (request, kv head)
 constexpr int kTileTokens = kPageSize * kPagesPerTile;
 constexpr int kMaxGroup = 8;         // query heads per KV head handled by one MMA column block
 constexpr int kMaxSpans = 2048;      // upper bound on the partition width (one span per warp)
@@ -363,7 +366,8 @@ struct AttnParams {
     float *part_ml;                 // [2*kMaxSpans][16]  (m[8], l[8])
     int32_t *arrivals;              // [kMaxSpans], all zero between launches
     int4 *span_start;               // [kMaxSpans] what each span started at (diagnostic)
-    unsigned long long *trace;      // [kMaxSpans][4] ns: start, first tile landed, last tile done, span done
+    unsigned long long *trace;      // [kMaxSpans][8] ns: start, first tile landed, last tile done, span done,
+                                    //   total wait for data, total time between pieces, tiles, pieces
     uint32_t *status;
     int32_t batch, max_pages_per_req, num_pages, num_kv_heads, num_q_heads, group;
     int32_t layer_page_base;        // layer * num_pages
@@ -521,10 +525,10 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     if (st.r < 0) {
         if (lane == 0) {
             p.span_start[span] = make_int4(-1, -1, -1, -1);
-            p.trace[span * 4 + 0] = t_start;
-            p.trace[span * 4 + 1] = 0;
+            p.trace[span * 8 + 0] = t_start;
+            p.trace[span * 8 + 1] = 0;
         }
-        if (lane == 0) p.trace[span * 4 + 2] = p.trace[span * 4 + 3] = global_timer_ns();
+        if (lane == 0) p.trace[span * 8 + 2] = p.trace[span * 8 + 3] = global_timer_ns();
         return;
     }
     const int n_total = st.count;
@@ -563,7 +567,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     };
 
     // Issue the loads of the tile under the issue cursor into stage issued % NS, then advance.
+#ifdef CKV_TRACE_WAITS
+    unsigned long long t_issue = 0, t_masked = 0;
+#endif
     auto issue_next = [&]() {
+#ifdef CKV_TRACE_WAITS
+        const unsigned long long i0 = global_timer_ns();
+#endif
         const int ck = ic.tile / kTilesPerChunk;
         if (ck != cur_chunk) {
             cur_chunk = ck;
@@ -575,8 +585,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         const int pg = lane / Lay::kHalves, hf = lane % Lay::kHalves;
         int page = __shfl_sync(0xffffffffu, cur_val, ((ic.tile % kTilesPerChunk) * kPagesPerTile + pg) & 31);
         const int slot = issued % NS;
-        fence_proxy_async();                      // this warp's earlier reads of the stage precede the copy
-        __syncwarp();
+        // The stage's previous contents were read by this warp's ldmatrix instructions, whose results
+        // have all been consumed by MMAs earlier in program order, so the reads are complete.
         if (lane == 0) mbar_arrive_expect_tx(bars + slot * 8, np * Lay::kPageBytes);
         __syncwarp();
         if (lane < np * Lay::kHalves) {
@@ -604,13 +614,16 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 }
             }
         }
+#ifdef CKV_TRACE_WAITS
+        t_issue += global_timer_ns() - i0;
+#endif
     };
 
     grid_dependency_wait();                       // the pool, the workspace and `out` are ours from here on
     if (lane == 0) {
         p.span_start[span] = make_int4(st.r, st.h, st.tile, st.begin);
-        p.trace[span * 4 + 0] = t_start;
-        p.trace[span * 4 + 1] = 0;
+        p.trace[span * 8 + 0] = t_start;
+        p.trace[span * 8 + 1] = 0;
     }
     for (int k = 0; k < NS && k < n_total; ++k) issue_next();
 
@@ -634,6 +647,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     int done = 0;                                // tiles computed (or skipped after a wait gave up)
     int landed = 0;                              // tiles whose copies were seen to complete
     long long t_global = st.begin;               // global index of the compute cursor's tile
+    unsigned long long t_wait = 0, t_between = 0, t_piece_end = 0;
+    int n_pieces = 0;
     bool first_piece = true;
     // a span writes at most two partials: its first piece and its last piece
     int pend_first[2] = {-1, -1}, pend_last[2] = {0, 0}, pend_slot[2] = {0, 0};
@@ -643,6 +658,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         const bool complete = (cc.tile == 0 && n == cc.tiles);
         const int piece_r = cc.r, piece_h = cc.h, piece_L = cc.L, piece_tile0 = cc.tile, piece_tiles = cc.tiles;
 
+        ++n_pieces;
         uint32_t qf[Lay::kKSteps][2];
         if (qn_r == piece_r && qn_h == piece_h) {
 #pragma unroll
@@ -659,12 +675,21 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         for (int ti = piece_tile0; ti < piece_tile0 + n; ++ti, ++done) {
             const int slot = done % NS;
             if (alive) {
+#ifdef CKV_TRACE_WAITS
+                const unsigned long long w0 = global_timer_ns();
+#endif
                 alive = mbar_wait_bounded(bars + slot * 8, (done / NS) & 1, p.status);
                 alive = __all_sync(0xffffffffu, alive);
+#ifdef CKV_TRACE_WAITS
+                t_wait += global_timer_ns() - w0;
+#endif
             }
             if (!alive) continue;
+#ifdef CKV_TRACE_WAITS
+            const unsigned long long w1 = global_timer_ns();
+#endif
             ++landed;
-            if (done == 0 && lane == 0) p.trace[span * 4 + 1] = global_timer_ns();
+            if (done == 0 && lane == 0) p.trace[span * 8 + 1] = global_timer_ns();
 
             const int ntok = min(kTileTokens, piece_L - ti * kTileTokens);      // valid tokens in this tile
             const bool full_tile = (ntok == kTileTokens);
@@ -683,6 +708,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                                        (16 + row0 + rem / 8) * 128 + (rem % 8) * 16;
                     asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
                 }
+                fence_proxy_async();              // these generic-proxy writes precede the stage's next TMA fill
                 __syncwarp();
             }
 
@@ -751,10 +777,14 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     }
                 }
             }
+#ifdef CKV_TRACE_WAITS
+            if (!full_tile) t_masked += global_timer_ns() - w1;
+#endif
             // the stage is free again: refill it with the tile NS ahead
             if (issued < n_total) issue_next();
         }
-        if (lane == 0 && done == n_total) p.trace[span * 4 + 2] = global_timer_ns();
+        if (lane == 0 && done == n_total) p.trace[span * 8 + 2] = global_timer_ns();
+        t_piece_end = global_timer_ns();
 
         // ---- finish the piece: row sums across the warp, then through the staging tile
 #pragma unroll
@@ -808,6 +838,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             pend_out[k] = out_rows;
         }
         __syncwarp();                             // staging is reused by the next piece
+        t_between += global_timer_ns() - t_piece_end;
         first_piece = false;
         t_global += n;
         if (done < n_total) {
@@ -839,7 +870,18 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     if (!alive) {
         for (int k = landed; k < issued; ++k) mbar_wait_bounded(bars + (k % NS) * 8, (k / NS) & 1, p.status);
     }
-    if (lane == 0) p.trace[span * 4 + 3] = global_timer_ns();
+    if (lane == 0) {
+        p.trace[span * 8 + 3] = global_timer_ns();
+        p.trace[span * 8 + 4] = t_wait;
+        p.trace[span * 8 + 5] = t_between;
+#ifdef CKV_TRACE_WAITS
+        p.trace[span * 8 + 6] = t_issue;
+        p.trace[span * 8 + 7] = t_masked;
+#else
+        p.trace[span * 8 + 6] = n_total;
+        p.trace[span * 8 + 7] = n_pieces;
+#endif
+    }
 }
 
 }  // namespace ckv

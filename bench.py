@@ -3,8 +3,8 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-sweep]
 
-One step = one pass of the whole hot path (append, split-KV plan, partial attention, combine) for
-every layer of the workload over one seeded synthetic batch.  The headline workload is the
+One step = one pass of the whole hot path (append, split-KV plan, partial attention, combine; one
+fused kernel per layer) for every layer of the workload over one seeded synthetic batch.  The headline workload is the
 Llama-3-8B-shaped layer at batch 64 with contexts uniform in [512, 4096] ("llama8b_b64",
 ~600 MB of KV per step, several times the L2 size, so every step streams from HBM).
 
@@ -127,17 +127,16 @@ class DeviceWorkload:
         self.bytes = wl.algorithmic_bytes(w, self.lens)
 
     def step_calls(self):
-        """Pre-marshalled (function, args) pairs of one step, so the timed loop is two C calls per layer."""
+        """Pre-marshalled (function, args) pairs of one step, so the timed loop is one C call per layer."""
         import torch
         from paper_2501_08090_b200 import binding
         lib, h = binding.lib, self.kp._h
         s = torch.cuda.current_stream().cuda_stream
         calls = []
         for layer in range(self.w.num_layers):
-            calls.append((lib.kv_append, (h, layer, self.B, self.bt.data_ptr(), self.sl.data_ptr(),
-                                          self.k_new[layer].data_ptr(), self.v_new[layer].data_ptr(), s)))
-            calls.append((lib.decode_attention, (h, layer, self.B, self.bt.data_ptr(), self.sl.data_ptr(),
-                                                 self.q[layer].data_ptr(), self.out[layer].data_ptr(), s)))
+            calls.append((lib.decode_step, (h, layer, self.B, self.bt.data_ptr(), self.sl.data_ptr(),
+                                            self.q[layer].data_ptr(), self.k_new[layer].data_ptr(),
+                                            self.v_new[layer].data_ptr(), self.out[layer].data_ptr(), s)))
         return calls
 
     def run_steps(self, n: int) -> None:
@@ -336,10 +335,10 @@ def run_ours(args) -> None:
     dw.run_steps(P)
     attn_ms, attn_n = dw.kp.profile_read()
     dw.kp.profile_enable(False)
-    attn_bytes = (dw.bytes["kv"] + dw.bytes["q_out"] + dw.bytes["tables"]) // w.num_layers
+    attn_bytes = dw.bytes["total"] // w.num_layers            # the fused kernel moves all of a step's bytes
     peak, peak_kind = measured_peak_gbs()
     achieved = attn_bytes / (attn_ms / attn_n * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "paged_decode_attn_kernel", "achieved": achieved, "peak": peak,
+    roofline = {"bound": "hbm", "kernel": "paged_decode_attn_kernel (fused append + plan + attention + combine)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": "of " + peak_kind,
                 "traffic": None, "bytes_per_launch": attn_bytes, "us_per_launch": attn_ms / attn_n * 1e3,
                 "frac_of_8TBs": achieved / (NORMALISED_TO_TBS * 1e3)}

@@ -118,15 +118,29 @@ int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch,
                          const void *d_q, void *d_out, void *stream);
 
 /*
+ * One layer's whole decode iteration in ONE kernel: kv_append and decode_attention fused.  The warp
+ * that processes the last tile of a (request, KV head) stores that pair's new key and value rows
+ * to the pool (bit-exactly what kv_append writes) and patches them into its staged tile, so the
+ * result equals kv_append followed by decode_attention (Section 2.1 "Inference Primer": each new
+ * token attends to all previous tokens' keys and values, its own included, and its key/value
+ * are cached).  Arguments as in those two calls.  Errors: CKV_EINVAL, CKV_ECUDA.
+ */
+int32_t decode_step(ckv_pool *pool, int32_t layer, int32_t batch,
+                    const int32_t *d_block_tables, const int32_t *d_seq_lens,
+                    const void *d_q, const void *d_k_new, const void *d_v_new, void *d_out,
+                    void *stream);
+
+/*
  * The split-KV partition decode_attention uses for these lengths, copied to the host for
  * inspection (runs a small kernel and synchronises `stream`; decode_attention itself derives the
  * same partition inside its attention kernel and launches no plan kernel).  A "tile" is 32
- * consecutive tokens of one (request, KV head); tiles are numbered request-major, then KV head,
- * then position, and span s -- the work of one warp -- owns tiles
- * [s*tiles_per_span, min((s+1)*tiles_per_span, total_tiles)).
- *   h_header[4]   : total_tiles, tiles_per_span, num_spans, num_spans_with_work
+ * consecutive tokens of one (request, KV head).  Work is laid out on an axis of units,
+ * request-major then KV head: each (request, KV head) contributes CKV_PIECE_COST_TILES (2)
+ * overhead units followed by one unit per tile.  Span s -- the work of one warp -- owns the tiles
+ * whose units fall in [s*units_per_span, min((s+1)*units_per_span, total_units)).
+ *   h_header[4]   : total_units, units_per_span, num_spans, number of spans with a non-empty range
  *   h_span_start  : int32 [num_spans][4] = request, kv head, first tile within that
- *                   (request, kv head), global index of the span's first tile; -1s if idle
+ *                   (request, kv head), unit index of that tile; -1s if the span holds no tile
  * h_span_start must hold 4*ckv_get_partition() ints.  Errors: CKV_EINVAL, CKV_ECUDA.
  */
 int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *stream,
@@ -155,7 +169,7 @@ int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits);
 
 /*
  * One whole iteration for one layer with HOST buffers (pinned memory recommended): copies the
- * tables, lengths, q, k_new and v_new to the device, runs kv_append and decode_attention, copies
+ * tables, lengths, q, k_new and v_new to the device, runs decode_step, copies
  * the output back and synchronises `stream`.  h_out: bf16 [batch][num_q_heads][head_dim].
  * Errors: as kv_append / decode_attention.
  */
@@ -168,8 +182,8 @@ int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch,
  * Iteration latency against batch size: the curve Algorithm 1 reads as ITL(batch size)
  * (Section 2.1, figure "Variation in inter-token latency and token throughput with
  * increasing batch size"; Section 4.1).  For each i < n_sizes, runs `warmup` untimed and `iters` timed
- * steps on the first batch_sizes[i] requests of the given arrays; a step is kv_append +
- * decode_attention for every layer.  Per-layer inputs are laid out
+ * steps on the first batch_sizes[i] requests of the given arrays; a step is decode_step (append
+ * + attention in one kernel) for every layer.  Per-layer inputs are laid out
  *   d_q, d_out [num_layers][batch_stride][Hq][d],  d_k_new, d_v_new [num_layers][batch_stride][Hkv][d].
  * Each timed step is bracketed by CUDA events on `stream`; if d_flush is not NULL,
  * flush_bytes of it are overwritten before every step (outside the timed bracket) so that no

@@ -18,13 +18,14 @@ LIBRARY = os.path.join(_HERE, "libchiron_kv.so")
 
 CKV_OK, CKV_EINVAL, CKV_ENOMEM, CKV_ECUDA, CKV_EBOUNDS, CKV_ETIMEOUT = 0, -1, -2, -3, -4, -5
 STATUS_BAD_LENGTH, STATUS_BAD_PAGE, STATUS_WAIT_LIMIT = 1, 2, 4
+TILE_TOKENS, PIECE_COST_TILES = 32, 2      # the plan's tile size and per-piece overhead units
 
 EXPORTS = (
     "kv_pool_bytes", "kv_workspace_bytes", "kv_pool_create", "kv_pool_destroy", "kv_append",
     "decode_attention", "decode_plan", "ckv_set_partition", "ckv_get_partition", "kv_check_status",
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
     "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace", "ckv_set_overlap",
-    "decode_attention_noalloc",
+    "decode_attention_noalloc", "decode_step",
 )
 
 
@@ -55,6 +56,7 @@ def _load() -> ctypes.CDLL:
     lib.kv_pool_destroy.restype = i32; lib.kv_pool_destroy.argtypes = [vp]
     lib.kv_append.restype = i32; lib.kv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.decode_attention.restype = i32; lib.decode_attention.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+    lib.decode_step.restype = i32; lib.decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.decode_plan.restype = i32; lib.decode_plan.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_set_partition.restype = i32; lib.ckv_set_partition.argtypes = [vp, i32]
     lib.ckv_set_overlap.restype = i32; lib.ckv_set_overlap.argtypes = [vp, i32]
@@ -170,6 +172,14 @@ class KvPool:
                                     _dev_ptr(seq_lens, torch.int32), _dev_ptr(q, torch.bfloat16),
                                     _dev_ptr(out, torch.bfloat16), _stream_ptr(stream)))
 
+    def decode_step(self, layer: int, block_tables, seq_lens, q, k_new, v_new, out, stream=None) -> None:
+        """kv_append + decode_attention of one layer in a single kernel."""
+        batch = int(seq_lens.shape[0])
+        _check(lib.decode_step(self._h, layer, batch, _dev_ptr(block_tables, torch.int32),
+                               _dev_ptr(seq_lens, torch.int32), _dev_ptr(q, torch.bfloat16),
+                               _dev_ptr(k_new, torch.bfloat16), _dev_ptr(v_new, torch.bfloat16),
+                               _dev_ptr(out, torch.bfloat16), _stream_ptr(stream)))
+
     def decode_plan(self, seq_lens, stream=None):
         """(header dict, int32 [num_spans][4] array of span starts)."""
         batch = int(seq_lens.shape[0])
@@ -177,7 +187,7 @@ class KvPool:
         starts = np.zeros((self.get_partition(), 4), dtype=np.int32)
         _check(lib.decode_plan(self._h, batch, _dev_ptr(seq_lens, torch.int32), _stream_ptr(stream),
                                header.ctypes.data, starts.ctypes.data))
-        keys = ("total_tiles", "tiles_per_span", "num_spans", "spans_with_work")
+        keys = ("total_units", "units_per_span", "num_spans", "spans_with_units")
         return dict(zip(keys, header.tolist())), starts
 
     def set_partition(self, num_spans: int) -> None:

@@ -373,12 +373,16 @@ int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d
     return CKV_OK;
 }
 
-int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
-                         const int32_t *d_seq_lens, const void *d_q, void *d_out, void *stream)
+// Attention for one layer, optionally with the KV append folded into the same kernel.
+static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, int32_t batch,
+                                const int32_t *d_block_tables, const int32_t *d_seq_lens, const void *d_q,
+                                const void *d_k_new, const void *d_v_new, void *d_out, void *stream)
 {
-    if (int32_t rc = check_call(pool, layer, batch, "decode_attention")) return rc;
-    if (!d_block_tables || !d_seq_lens || !d_q || !d_out) return fail(CKV_EINVAL, "decode_attention: NULL argument");
-    if (!aligned16(d_q) || !aligned16(d_out)) return fail(CKV_EINVAL, "decode_attention: q/out not 16-byte aligned");
+    if (int32_t rc = check_call(pool, layer, batch, fn)) return rc;
+    if (!d_block_tables || !d_seq_lens || !d_q || !d_out) return fail(CKV_EINVAL, "%s: NULL argument", fn);
+    if (!aligned16(d_q) || !aligned16(d_out)) return fail(CKV_EINVAL, "%s: q/out not 16-byte aligned", fn);
+    if ((d_k_new == nullptr) != (d_v_new == nullptr)) return fail(CKV_EINVAL, "%s: k_new and v_new go together", fn);
+    if (d_k_new && (!aligned16(d_k_new) || !aligned16(d_v_new))) return fail(CKV_EINVAL, "%s: k_new/v_new not 16-byte aligned", fn);
     const ckv_config &c = pool->cfg;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
@@ -387,6 +391,10 @@ int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int
     ap.seq_lens = d_seq_lens;
     ap.q = static_cast<const uint16_t *>(d_q);
     ap.out = static_cast<uint16_t *>(d_out);
+    ap.k_new = static_cast<const uint4 *>(d_k_new);
+    ap.v_new = static_cast<const uint4 *>(d_v_new);
+    ap.pool_layer = d_k_new ? reinterpret_cast<uint4 *>(pool->d_pool + (size_t)c.num_pages * c.num_kv_heads * 2 * c.page_size * c.head_dim * 2 * layer)
+                            : nullptr;
     ap.part_acc = pool->wsp<float>(pool->ws.part_acc);
     ap.part_ml = pool->wsp<float>(pool->ws.part_ml);
     ap.arrivals = pool->wsp<int32_t>(pool->ws.arrivals);
@@ -424,6 +432,22 @@ int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int
     if (ev1) CKV_CUDA(cudaEventRecord(ev1, s));
     pool->launches += 1;
     return CKV_OK;
+}
+
+int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
+                         const int32_t *d_seq_lens, const void *d_q, void *d_out, void *stream)
+{
+    return attention_launch(pool, "decode_attention", layer, batch, d_block_tables, d_seq_lens, d_q, nullptr, nullptr,
+                            d_out, stream);
+}
+
+int32_t decode_step(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
+                    const int32_t *d_seq_lens, const void *d_q, const void *d_k_new, const void *d_v_new,
+                    void *d_out, void *stream)
+{
+    if (!d_k_new || !d_v_new) return fail(CKV_EINVAL, "decode_step: NULL k_new/v_new");
+    return attention_launch(pool, "decode_step", layer, batch, d_block_tables, d_seq_lens, d_q, d_k_new, d_v_new,
+                            d_out, stream);
 }
 
 int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *stream,
@@ -479,8 +503,7 @@ int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch, const int
     CKV_CUDA(cudaMemcpyAsync(d_q, h_q, (size_t)batch * c.num_q_heads * d2, cudaMemcpyHostToDevice, s));
     CKV_CUDA(cudaMemcpyAsync(d_k, h_k_new, (size_t)batch * c.num_kv_heads * d2, cudaMemcpyHostToDevice, s));
     CKV_CUDA(cudaMemcpyAsync(d_v, h_v_new, (size_t)batch * c.num_kv_heads * d2, cudaMemcpyHostToDevice, s));
-    if (int32_t rc = kv_append(pool, layer, batch, d_bt, d_sl, d_k, d_v, stream)) return rc;
-    if (int32_t rc = decode_attention(pool, layer, batch, d_bt, d_sl, d_q, d_o, stream)) return rc;
+    if (int32_t rc = decode_step(pool, layer, batch, d_bt, d_sl, d_q, d_k, d_v, d_o, stream)) return rc;
     CKV_CUDA(cudaMemcpyAsync(h_out, d_o, (size_t)batch * c.num_q_heads * d2, cudaMemcpyDeviceToHost, s));
     CKV_CUDA(cudaStreamSynchronize(s));
     return CKV_OK;
@@ -523,8 +546,7 @@ int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch
                 const uint8_t *kn = static_cast<const uint8_t *>(d_k_new) + kv_layer * layer;
                 const uint8_t *vn = static_cast<const uint8_t *>(d_v_new) + kv_layer * layer;
                 uint8_t *o = static_cast<uint8_t *>(d_out) + q_layer * layer;
-                rc = kv_append(pool, layer, b, d_block_tables, d_seq_lens, kn, vn, stream);
-                if (rc == CKV_OK) rc = decode_attention(pool, layer, b, d_block_tables, d_seq_lens, q, o, stream);
+                rc = decode_step(pool, layer, b, d_block_tables, d_seq_lens, q, kn, vn, o, stream);
             }
             if (timed) cudaEventRecord(ev[2 * (size_t)(k - warmup) + 1], s);
         }

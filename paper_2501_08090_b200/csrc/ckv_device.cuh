@@ -27,13 +27,21 @@ constexpr uint32_t kStatusWaitLimit = 4u;
 
 constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // bound of every device-side wait
 
-// The split-KV partition.  Tiles of all (request, kv head) pairs are numbered request-major, then
-// kv head, then position; span s owns tiles [s*q, min((s+1)*q, total)) with q = ceil(total/spans).
+// The split-KV partition.  Work is laid out on one axis of "units", request-major, then kv head:
+// every (request, kv head) contributes kPieceCostTiles overhead units (the fixed cost of starting,
+// finishing and merging a piece, measured at about two tiles' worth of time) followed by one unit
+// per tile.  Span s owns the tiles whose units fall in [s*q, min((s+1)*q, total)), q =
+// ceil(total/spans), so spans that hold many short (request, kv head) pieces get fewer tiles.
+#ifndef CKV_PIECE_COST_TILES
+#define CKV_PIECE_COST_TILES 2
+#endif
+constexpr int kPieceCostTiles = CKV_PIECE_COST_TILES;
+
 struct PlanHeader {
-    int32_t total_tiles;
-    int32_t tiles_per_span;
+    int32_t total_units;
+    int32_t units_per_span;
     int32_t num_spans;
-    int32_t spans_with_work;
+    int32_t spans_with_units;
 };
 
 // A context length is usable if 1 <= L <= table capacity; otherwise the request has no tiles.
@@ -100,11 +108,11 @@ __global__ void kv_append_kernel(const AppendParams p)
 // partition for every span at once, for inspection through decode_plan().
 // ------------------------------------------------------------------------------------------
 struct SpanStart {
-    int r, h, tile;        // first tile of the span: request, kv head, tile within (r, h); r = -1: no work
+    int r, h, tile;        // first tile of the span: request, kv head, tile within (r, h); r = -1: no tile
     int tiles_r;           // tiles per kv head of request r
     int L;                 // context length of request r
-    int count;             // tiles in the span
-    int begin;             // global index of the span's first tile
+    long long v;           // unit index of that first tile
+    long long end;         // one past the span's last unit
     int total, q;          // header values
 };
 
@@ -128,8 +136,11 @@ __device__ __forceinline__ void flag_unusable_requests(const int32_t *__restrict
     }
 }
 
-// Executed by one whole warp.  Two passes over seq_lens: the total, then the request that holds
-// tile span*q.
+// Units of one kv head of a request with t tiles (0 if the request is unusable).
+__device__ __forceinline__ int units_of_tiles(int t) { return t > 0 ? t + kPieceCostTiles : 0; }
+
+// Executed by one whole warp.  Two passes over seq_lens: the total number of units, then the
+// (request, kv head) that holds unit span*q and the first tile at or after it.
 __device__ __forceinline__ SpanStart warp_plan(const int32_t *__restrict__ seq_lens, int batch, int max_pages_per_req,
                                                int num_kv_heads, int num_spans, int span, int lane)
 {
@@ -137,41 +148,44 @@ __device__ __forceinline__ SpanStart warp_plan(const int32_t *__restrict__ seq_l
     int sum = 0;
     for (int base = 0; base < batch; base += 32) {
         const int r = base + lane;
-        if (r < batch) {
-            sum += tiles_of_length(__ldg(seq_lens + r), max_pages_per_req);
-        }
+        if (r < batch) sum += units_of_tiles(tiles_of_length(__ldg(seq_lens + r), max_pages_per_req));
     }
 #pragma unroll
     for (int x = 16; x > 0; x >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, x);
     s.total = sum * num_kv_heads;
     s.q = max(1, (s.total + num_spans - 1) / num_spans);
     const long long begin = (long long)span * s.q;
-    s.r = -1; s.h = s.tile = s.tiles_r = s.L = s.count = 0;
-    s.begin = (int)min(begin, (long long)s.total);
+    s.r = -1; s.h = s.tile = s.tiles_r = s.L = 0;
+    s.v = s.end = min(begin, (long long)s.total);
     if (begin >= s.total) return s;
-    s.count = (int)min((long long)s.q, (long long)s.total - begin);
+    s.end = min(begin + s.q, (long long)s.total);
 
-    long long running = 0;                               // tiles (all heads) before request `base`
+    long long running = 0;                               // units (all heads) before request `base`
     for (int base = 0; base < batch; base += 32) {
         const int r = base + lane;
         const int L = r < batch ? __ldg(seq_lens + r) : 0;
         const int t = r < batch ? tiles_of_length(L, max_pages_per_req) : 0;
-        int incl = t;
+        int incl = units_of_tiles(t);
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const int v = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += v;
         }
-        const long long upto = running + (long long)incl * num_kv_heads;     // tiles through request r
+        const long long upto = running + (long long)incl * num_kv_heads;     // units through request r
         const unsigned hit = __ballot_sync(0xffffffffu, upto > begin);
         if (hit) {
             const int src = __ffs(hit) - 1;
             const int t_r = __shfl_sync(0xffffffffu, t, src);
             const int L_r = __shfl_sync(0xffffffffu, L, src);
-            const long long before = __shfl_sync(0xffffffffu, upto, src) - (long long)t_r * num_kv_heads;
+            const int u_r = t_r + kPieceCostTiles;
+            const long long before = __shfl_sync(0xffffffffu, upto, src) - (long long)u_r * num_kv_heads;
             const int rem = (int)(begin - before);
+            const int h = rem / u_r, off = rem % u_r;
+            const int tile = max(0, off - kPieceCostTiles);               // a span starting in the overhead
+            const long long v = before + (long long)h * u_r + kPieceCostTiles + tile;   // units starts at tile 0
+            if (v >= s.end) return s;                                      // the span holds overhead units only
             s.r = base + src; s.tiles_r = t_r; s.L = L_r;
-            s.h = rem / t_r; s.tile = rem % t_r;
+            s.h = h; s.tile = tile; s.v = v;
             return s;
         }
         running = __shfl_sync(0xffffffffu, upto, 31);
@@ -182,7 +196,7 @@ __device__ __forceinline__ SpanStart warp_plan(const int32_t *__restrict__ seq_l
 struct PlanParams {
     const int32_t *seq_lens;
     PlanHeader *header;
-    int4 *span_start;               // [num_spans] request, kv head, tile, global tile index (-1s if idle)
+    int4 *span_start;               // [num_spans] request, kv head, tile, unit index of that tile (-1s if idle)
     int32_t batch, max_pages_per_req, num_kv_heads, num_spans;
 };
 
@@ -193,12 +207,12 @@ __global__ void splitkv_plan_kernel(const PlanParams p)
     for (int span = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; span < p.num_spans; span += warps) {
         const SpanStart s = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane);
         if (lane == 0) {
-            p.span_start[span] = s.r < 0 ? make_int4(-1, -1, -1, -1) : make_int4(s.r, s.h, s.tile, s.begin);
+            p.span_start[span] = s.r < 0 ? make_int4(-1, -1, -1, -1) : make_int4(s.r, s.h, s.tile, (int)s.v);
             if (span == 0) {
-                p.header->total_tiles = s.total;
-                p.header->tiles_per_span = s.q;
+                p.header->total_units = s.total;
+                p.header->units_per_span = s.q;
                 p.header->num_spans = p.num_spans;
-                p.header->spans_with_work = (s.total + s.q - 1) / s.q;
+                p.header->spans_with_units = (s.total + s.q - 1) / s.q;
             }
         }
     }
@@ -352,6 +366,12 @@ __device__ __forceinline__ float4 ld_cg_f32x4(const float *p)
 // The S^T accumulator fragment holds (token = lane/4 [+8], g = 2*(lane%4)+{0,1}); packed to bf16
 // and transposed with movmatrix it is exactly the B fragment of P^T.
 //
+// Fused append (k_new != NULL): the warp whose span holds the LAST tile of a (request, kv head)
+// owns that pair's append.  It stores the new key and value rows to the pool for later
+// iterations, and overwrites the same rows of its staged tile in shared memory before computing
+// on it -- so this iteration sees the new token whether the tile's copy read the pool before or
+// after the store landed.  No other warp reads that slot as a live token in this launch.
+//
 // A piece is the part of one (request, kv head) that falls inside the span.  When it covers the
 // whole context the warp normalises and writes the bf16 output rows itself.  Otherwise it stores
 // an fp32 partial (m, l, O) and bumps an arrival counter; whichever warp arrives last for that
@@ -362,6 +382,10 @@ struct AttnParams {
     const int32_t *seq_lens;
     const uint16_t *q;
     uint16_t *out;
+    // fused KV append (all three NULL for attention alone): the new token's rows and this layer's pool slice
+    const uint4 *k_new;             // bf16 [batch][Hkv][d]
+    const uint4 *v_new;
+    uint4 *pool_layer;
     float *part_acc;                // [2*kMaxSpans][8][D]
     float *part_ml;                 // [2*kMaxSpans][16]  (m[8], l[8])
     int32_t *arrivals;              // [kMaxSpans], all zero between launches
@@ -386,17 +410,23 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
     const int pieces = s_last - s_first + 1;
     auto slot_of = [&](int i) { return i == 0 ? slot_first : 2 * (s_first + i); };
 
+    // (m, l) of the partial this lane owns in the first round of 32; usually the only round
+    float mi[kMaxGroup], li[kMaxGroup];
+    auto load_ml = [&](int i) {
+        const float *ml = part_ml + slot_of(i) * 2 * kMaxGroup;
+        const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
+        const float4 c = ld_cg_f32x4(ml + 8), d = ld_cg_f32x4(ml + 12);
+        mi[0] = a.x; mi[1] = a.y; mi[2] = a.z; mi[3] = a.w; mi[4] = b.x; mi[5] = b.y; mi[6] = b.z; mi[7] = b.w;
+        li[0] = c.x; li[1] = c.y; li[2] = c.z; li[3] = c.w; li[4] = d.x; li[5] = d.y; li[6] = d.z; li[7] = d.w;
+    };
     float mstar[kMaxGroup];
 #pragma unroll
     for (int g = 0; g < kMaxGroup; ++g) mstar[g] = -INFINITY;
-    for (int base = 0; base < pieces; base += 32) {
+    for (int base = (pieces - 1) & ~31; base >= 0; base -= 32) {       // round 0 last: its values stay in mi, li
         if (base + lane < pieces) {
-            const float *ml = part_ml + slot_of(base + lane) * 2 * kMaxGroup;
-            const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
-            mstar[0] = fmaxf(mstar[0], a.x); mstar[1] = fmaxf(mstar[1], a.y);
-            mstar[2] = fmaxf(mstar[2], a.z); mstar[3] = fmaxf(mstar[3], a.w);
-            mstar[4] = fmaxf(mstar[4], b.x); mstar[5] = fmaxf(mstar[5], b.y);
-            mstar[6] = fmaxf(mstar[6], b.z); mstar[7] = fmaxf(mstar[7], b.w);
+            load_ml(base + lane);
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g) mstar[g] = fmaxf(mstar[g], mi[g]);
         }
     }
 #pragma unroll
@@ -414,11 +444,7 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
 #pragma unroll
         for (int g = 0; g < kMaxGroup; ++g) f_mine[g] = 0.f;
         if (base + lane < pieces) {
-            const float *ml = part_ml + slot_of(base + lane) * 2 * kMaxGroup;
-            const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
-            const float4 c = ld_cg_f32x4(ml + 8), d = ld_cg_f32x4(ml + 12);
-            const float mi[kMaxGroup] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-            const float li[kMaxGroup] = {c.x, c.y, c.z, c.w, d.x, d.y, d.z, d.w};
+            if (base > 0) load_ml(base + lane);
 #pragma unroll
             for (int g = 0; g < kMaxGroup; ++g) {
                 f_mine[g] = fast_exp2(mi[g] - mstar[g]);
@@ -472,12 +498,15 @@ struct AttnLayout {
 struct SpanCursor {
     int r, h, tile;       // next tile: request, kv head, tile within (r, h)
     int L, tiles;         // length and tile count of request r
+    long long v;          // unit index of that tile on the plan's axis
 
     // step to the next tile; returns false when it left the last request
     __device__ __forceinline__ bool next(const AttnParams &p)
     {
+        ++v;
         if (++tile < tiles) return true;
         tile = 0;
+        v += kPieceCostTiles;                 // the next (request, kv head) starts with its overhead units
         if (++h < p.num_kv_heads) return true;
         h = 0;
         do {
@@ -531,13 +560,14 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         if (lane == 0) p.trace[span * 8 + 2] = p.trace[span * 8 + 3] = global_timer_ns();
         return;
     }
-    const int n_total = st.count;
+    const long long v_end = st.end;
     const int q_span = st.q;
     const int G = p.group;
 
     // ---- issue side: block-table entries travel in registers, 32 pages (16 tiles) per chunk
     SpanCursor ic;
-    ic.r = st.r; ic.h = st.h; ic.tile = st.tile; ic.L = st.L; ic.tiles = st.tiles_r;
+    ic.r = st.r; ic.h = st.h; ic.tile = st.tile; ic.L = st.L; ic.tiles = st.tiles_r; ic.v = st.v;
+    bool more_to_issue = true;                   // the issue cursor still points at a tile of this span
     int issued = 0;
     bool alive = true;
     auto table_row = [&](int r) { return p.block_tables + (size_t)r * p.max_pages_per_req; };
@@ -567,6 +597,16 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     };
 
     // Issue the loads of the tile under the issue cursor into stage issued % NS, then advance.
+    // rows of the (request, kv head) whose last tile is in flight: lane l < 2*d/8 holds 16 bytes of
+    // the key row (first d/8 lanes) or of the value row
+    constexpr int kRowVecs = D / 8;
+    uint4 an_val = make_uint4(0u, 0u, 0u, 0u);
+    int an_r = -1, an_h = -1, an_page = -1;
+    auto load_new_rows = [&](int r, int h) -> uint4 {
+        if (lane >= 2 * kRowVecs) return make_uint4(0u, 0u, 0u, 0u);
+        const uint4 *src = (lane < kRowVecs ? p.k_new : p.v_new) + ((size_t)r * p.num_kv_heads + h) * kRowVecs;
+        return __ldg(src + (lane % kRowVecs));
+    };
 #ifdef CKV_TRACE_WAITS
     unsigned long long t_issue = 0, t_masked = 0;
 #endif
@@ -590,17 +630,25 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         if (lane == 0) mbar_arrive_expect_tx(bars + slot * 8, np * Lay::kPageBytes);
         __syncwarp();
         if (lane < np * Lay::kHalves) {
+            int src_page = page;
             if (page < 0 || page >= p.num_pages) {
                 atomicOr(p.status, kStatusBadPage);
-                page = 0;
+                src_page = 0;
             }
-            const int y = ((p.layer_page_base + page) * p.num_kv_heads + ic.h) * 32;
+            const int y = ((p.layer_page_base + src_page) * p.num_kv_heads + ic.h) * 32;
             tma_load_2d(ring + slot * Lay::kStageBytes + pg * Lay::kPageBytes + hf * Lay::kHalfBytes,
                         &tmap, hf * 64, y, bars + slot * 8);
         }
+        if (p.k_new != nullptr && ic.tile == ic.tiles - 1 && an_r < 0) {
+            // last tile of this (request, kv head): fetch the rows to append and remember their page
+            const bool bad = page < 0 || page >= p.num_pages;               // before any redirect above
+            an_val = load_new_rows(ic.r, ic.h);
+            an_page = __shfl_sync(0xffffffffu, bad ? -1 : page, (np - 1) * Lay::kHalves);
+            an_r = ic.r; an_h = ic.h;
+        }
         ++issued;
-        if (issued < n_total) {
-            ic.next(p);
+        more_to_issue = ic.next(p) && ic.v < v_end;
+        if (more_to_issue) {
             if (ic.tile == 0) {
                 // entered a new (request, kv head): its first table chunk was fetched ahead
                 cur_chunk = 0;
@@ -621,15 +669,15 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 
     grid_dependency_wait();                       // the pool, the workspace and `out` are ours from here on
     if (lane == 0) {
-        p.span_start[span] = make_int4(st.r, st.h, st.tile, st.begin);
+        p.span_start[span] = make_int4(st.r, st.h, st.tile, (int)st.v);
         p.trace[span * 8 + 0] = t_start;
         p.trace[span * 8 + 1] = 0;
     }
-    for (int k = 0; k < NS && k < n_total; ++k) issue_next();
+    for (int k = 0; k < NS && more_to_issue; ++k) issue_next();
 
     // ---- compute side
     SpanCursor cc;
-    cc.r = st.r; cc.h = st.h; cc.tile = st.tile; cc.L = st.L; cc.tiles = st.tiles_r;
+    cc.r = st.r; cc.h = st.h; cc.tile = st.tile; cc.L = st.L; cc.tiles = st.tiles_r; cc.v = st.v;
     const int g0 = (lane & 3) * 2;               // first of the two group columns this lane accumulates
     uint32_t k_off[4], v_off[4];                 // ldmatrix lane offsets inside one page block
     {
@@ -646,15 +694,15 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 
     int done = 0;                                // tiles computed (or skipped after a wait gave up)
     int landed = 0;                              // tiles whose copies were seen to complete
-    long long t_global = st.begin;               // global index of the compute cursor's tile
+    bool more_to_compute = true;
     unsigned long long t_wait = 0, t_between = 0, t_piece_end = 0;
     int n_pieces = 0;
     bool first_piece = true;
     // a span writes at most two partials: its first piece and its last piece
     int pend_first[2] = {-1, -1}, pend_last[2] = {0, 0}, pend_slot[2] = {0, 0};
     uint16_t *pend_out[2] = {nullptr, nullptr};
-    while (done < n_total) {
-        const int n = min(cc.tiles - cc.tile, n_total - done);
+    while (more_to_compute) {
+        const int n = (int)min((long long)(cc.tiles - cc.tile), v_end - cc.v);
         const bool complete = (cc.tile == 0 && n == cc.tiles);
         const int piece_r = cc.r, piece_h = cc.h, piece_L = cc.L, piece_tile0 = cc.tile, piece_tiles = cc.tiles;
 
@@ -709,6 +757,34 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0u) : "memory");
                 }
                 fence_proxy_async();              // these generic-proxy writes precede the stage's next TMA fill
+                __syncwarp();
+            }
+
+            if (p.k_new != nullptr && ti == piece_tiles - 1) {
+                // this warp owns the append of (piece_r, piece_h): position L-1 is in the tile's last page
+                uint4 val;
+                int page;
+                if (an_r == piece_r && an_h == piece_h) {
+                    val = an_val; page = an_page; an_r = -1;
+                } else {                                                     // not fetched ahead (very short contexts)
+                    val = load_new_rows(piece_r, piece_h);
+                    page = __ldg(table_row(piece_r) + (piece_L - 1) / kPageSize);
+                    if (page < 0 || page >= p.num_pages) page = -1;
+                }
+                const int pos_slot = (piece_L - 1) % kPageSize;
+                if (lane < 2 * kRowVecs) {
+                    const int kv = lane / kRowVecs, vec = lane % kRowVecs;
+                    if (page >= 0) {
+                        const size_t row = (((size_t)page * p.num_kv_heads + piece_h) * 2 + kv) * kPageSize + pos_slot;
+                        p.pool_layer[row * kRowVecs + vec] = val;
+                    } else {
+                        atomicOr(p.status, kStatusBadPage);
+                    }
+                    const uint32_t a = sb + (np - 1) * Lay::kPageBytes + (vec / 8) * Lay::kHalfBytes +
+                                       (kv * 16 + pos_slot) * 128 + (((vec % 8) ^ (pos_slot & 7)) << 4);
+                    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(val.x), "r"(val.y), "r"(val.z), "r"(val.w) : "memory");
+                }
+                fence_proxy_async();              // generic-proxy writes precede the stage's next TMA fill
                 __syncwarp();
             }
 
@@ -778,12 +854,11 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 }
             }
 #ifdef CKV_TRACE_WAITS
-            if (!full_tile) t_masked += global_timer_ns() - w1;
+            if (ti == piece_tile0 && !first_piece) t_masked += global_timer_ns() - w1;
 #endif
             // the stage is free again: refill it with the tile NS ahead
-            if (issued < n_total) issue_next();
+            if (more_to_issue) issue_next();
         }
-        if (lane == 0 && done == n_total) p.trace[span * 8 + 2] = global_timer_ns();
         t_piece_end = global_timer_ns();
 
         // ---- finish the piece: row sums across the warp, then through the staging tile
@@ -829,40 +904,48 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             }
             // ---- remember the arrival; it is made once the whole span has been streamed, so that
             // neither the fence nor a merge ever interrupts this warp's loads
-            const long long item_begin = t_global - piece_tile0;
-            const long long item_end = item_begin + piece_tiles;
+            const long long tile0_unit = cc.v - piece_tile0;             // unit of this (request, kv head)'s tile 0
             const int k = first_piece ? 0 : 1;
-            pend_first[k] = (int)(item_begin / q_span);
-            pend_last[k] = (int)((item_end - 1) / q_span);
-            pend_slot[k] = (item_begin == (long long)pend_first[k] * q_span) ? 2 * pend_first[k] : 2 * pend_first[k] + 1;
+            pend_first[k] = (int)(tile0_unit / q_span);
+            pend_last[k] = (int)((tile0_unit + piece_tiles - 1) / q_span);
+            // in span pend_first the piece is that span's first one iff the span starts inside this
+            // (request, kv head)'s overhead units or exactly at them
+            pend_slot[k] = ((long long)pend_first[k] * q_span >= tile0_unit - kPieceCostTiles) ? 2 * pend_first[k]
+                                                                                              : 2 * pend_first[k] + 1;
             pend_out[k] = out_rows;
         }
         __syncwarp();                             // staging is reused by the next piece
         t_between += global_timer_ns() - t_piece_end;
         first_piece = false;
-        t_global += n;
-        if (done < n_total) {
-            // move the compute cursor to the start of the next (request, kv head)
-            cc.tile = cc.tiles - 1;
-            cc.next(p);
-        }
+        // move the compute cursor past the piece: to the next (request, kv head) or out of the span
+        cc.tile += n - 1;
+        cc.v += n - 1;
+        more_to_compute = cc.next(p) && cc.v < v_end;
     }
+
+    if (lane == 0) p.trace[span * 8 + 2] = global_timer_ns();
 
     // ---- arrivals: whichever warp arrives last for a (request, kv head) merges its partials (wait-free)
     if (pend_first[0] >= 0 || pend_first[1] >= 0) {
         __threadfence();
         __syncwarp();
-#pragma unroll
-        for (int k = 0; k < 2; ++k) {
-            if (pend_first[k] < 0) continue;
-            int prior = 0;
-            if (lane == 0) prior = atomicAdd(p.arrivals + pend_first[k], 1);
-            prior = __shfl_sync(0xffffffffu, prior, 0);
-            if (prior == pend_last[k] - pend_first[k]) {
-                __threadfence();
-                if (lane == 0) p.arrivals[pend_first[k]] = 0;        // ready for the next launch
-                combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k], pend_slot[k], G, lane);
+        int prior0 = 0, prior1 = 0;
+        if (lane == 0) {                          // both round trips in flight together
+            if (pend_first[0] >= 0) prior0 = atomicAdd(p.arrivals + pend_first[0], 1);
+            if (pend_first[1] >= 0) prior1 = atomicAdd(p.arrivals + pend_first[1], 1);
+        }
+        prior0 = __shfl_sync(0xffffffffu, prior0, 0);
+        prior1 = __shfl_sync(0xffffffffu, prior1, 0);
+        const bool last0 = pend_first[0] >= 0 && prior0 == pend_last[0] - pend_first[0];
+        const bool last1 = pend_first[1] >= 0 && prior1 == pend_last[1] - pend_first[1];
+        if (last0 || last1) {
+            __threadfence();
+            if (lane == 0) {                      // counters are ready for the next launch
+                if (last0) p.arrivals[pend_first[0]] = 0;
+                if (last1) p.arrivals[pend_first[1]] = 0;
             }
+            if (last0) combine_partials<D>(p.part_acc, p.part_ml, pend_out[0], pend_first[0], pend_last[0], pend_slot[0], G, lane);
+            if (last1) combine_partials<D>(p.part_acc, p.part_ml, pend_out[1], pend_first[1], pend_last[1], pend_slot[1], G, lane);
         }
     }
 
@@ -878,7 +961,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         p.trace[span * 8 + 6] = t_issue;
         p.trace[span * 8 + 7] = t_masked;
 #else
-        p.trace[span * 8 + 6] = n_total;
+        p.trace[span * 8 + 6] = done;
         p.trace[span * 8 + 7] = n_pieces;
 #endif
     }

@@ -106,3 +106,56 @@ def compact_requests(pool_dev: torch.Tensor, bt: np.ndarray, lens: np.ndarray, r
     ids = torch.from_numpy(np.concatenate(ids).astype(np.int64)).to(pool_dev.device)
     sub = pool_dev[layer].index_select(0, ids)
     return dev_to_bits(sub).reshape(-1), new_bt, lens[rows].astype(np.int32), at
+
+
+# ----------------------------------------------------------------------------- the plan's spec
+
+def expected_plan(lens_np, Hkv, C, cost=2):
+    """The partition spec restated: `cost` overhead units then one unit per 32-token tile for every
+    (request, kv head); span s owns the tiles whose units lie in [s*q, (s+1)*q)."""
+    tiles = (lens_np.astype(np.int64) + 31) // 32
+    units = tiles + cost
+    prefix = np.concatenate([[0], np.cumsum(units)]) * Hkv
+    total = int(prefix[-1])
+    q = max(1, -(-total // C))
+    starts = np.full((C, 4), -1, dtype=np.int64)
+    for c in range(C):
+        b0, e0 = c * q, min((c + 1) * q, total)
+        if b0 >= total:
+            continue
+        r = int(np.searchsorted(prefix, b0, side="right") - 1)
+        rem = b0 - int(prefix[r])
+        h, off = rem // int(units[r]), rem % int(units[r])
+        tile = max(0, off - cost)
+        v = int(prefix[r]) + h * int(units[r]) + cost + tile
+        if v < e0:
+            starts[c] = [r, h, tile, v]
+    return total, q, starts.astype(np.int32)
+
+
+def covered_tiles(lens_np, Hkv, C, cost=2, counts=None):
+    """All (request, kv head, tile) triples the spans of the spec visit, in order.
+    If `counts` is a list, the number of tiles of every span is appended to it."""
+    tiles = (lens_np.astype(np.int64) + 31) // 32
+    total, q, starts = expected_plan(lens_np, Hkv, C, cost)
+    seen = []
+    for c in range(C):
+        r, h, tile, v = (int(x) for x in starts[c])
+        before = len(seen)
+        if counts is not None:
+            counts.append(0)
+        if r < 0:
+            continue
+        end = min((c + 1) * q, total)
+        while v < end:
+            seen.append((r, h, tile))
+            v += 1; tile += 1
+            if tile == tiles[r]:
+                tile = 0; v += cost; h += 1
+                if h == Hkv:
+                    h = 0; r += 1
+                    if r == lens_np.size:
+                        break
+        if counts is not None:
+            counts[-1] = len(seen) - before
+    return seen

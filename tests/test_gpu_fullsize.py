@@ -114,8 +114,7 @@ def test_llama70b_all_80_layers_sampled_parity():
     refs = {layer: _oracle_on_sample(w, pool, bt, lens, rows, layer, q, k, v) for layer in layers}
     btd, sld = torch.from_numpy(bt).cuda(), torch.from_numpy(lens).cuda()
     for layer in range(w.num_layers):                                      # one whole decode iteration
-        kp.kv_append(layer, btd, sld, k[layer], v[layer])
-        kp.decode_attention(layer, btd, sld, q[layer], out[layer])
+        kp.decode_step(layer, btd, sld, q[layer], k[layer], v[layer], out[layer])
     assert kp.check_status() == 0
     assert torch.isfinite(out.float()).all()
     for layer in layers:

@@ -13,7 +13,7 @@ from oracle import oracle
 from oracle.oracle import PoolShape
 from paper_2501_08090_b200 import workloads as wl
 
-from helpers import (assert_close, bits_to_dev, dev_to_bits, make_device_step, oracle_step,
+from helpers import (assert_close, bits_to_dev, dev_to_bits, expected_plan, make_device_step, oracle_step,
                      pool_shape, widen)
 
 pytestmark = pytest.mark.gpu
@@ -24,12 +24,15 @@ def binding():
     return b
 
 
-def run_step(h, layer=0, partition=None):
+def run_step(h, layer=0, partition=None, fused=False):
     ds = make_device_step(h)
     if partition is not None:
         ds.pool.set_partition(partition)
-    ds.pool.kv_append(layer, ds.bt, ds.sl, ds.k_new[layer], ds.v_new[layer])
-    ds.pool.decode_attention(layer, ds.bt, ds.sl, ds.q[layer], ds.out[layer])
+    if fused:
+        ds.pool.decode_step(layer, ds.bt, ds.sl, ds.q[layer], ds.k_new[layer], ds.v_new[layer], ds.out[layer])
+    else:
+        ds.pool.kv_append(layer, ds.bt, ds.sl, ds.k_new[layer], ds.v_new[layer])
+        ds.pool.decode_attention(layer, ds.bt, ds.sl, ds.q[layer], ds.out[layer])
     bits = ds.pool.check_status()
     assert bits == 0
     return ds
@@ -65,6 +68,55 @@ def test_partition_invariance_on_tiny_workload(partition):
     _, ref_out = oracle_step(h)
     ds = run_step(h, partition=partition)
     assert_close(dev_to_bits(ds.out[0]), ref_out, "tiny/partition=%d" % partition)
+
+
+# --------------------------------------------------------------------------- fused append + attention
+
+@pytest.mark.parametrize("Hq,Hkv,d", [(4, 1, 64), (8, 2, 128), (32, 8, 128), (64, 8, 128), (5, 1, 128)])
+def test_decode_step_equals_append_then_attention(Hq, Hkv, d):
+    lens = [1, 2, 15, 16, 17, 31, 32, 33, 47, 48, 49, 64, 65, 96, 97, 129, 300, 1000, 2049]
+    h = custom_inputs(lens, Hq, Hkv, d, seed=Hq * 7 + d)
+    ref_pool, ref_out = oracle_step(h)
+    for partition in (None, 1, 9, 2048):
+        ds = run_step(h, partition=partition, fused=True)
+        assert np.array_equal(dev_to_bits(ds.pool.pool), ref_pool)           # every byte of the pool
+        assert_close(dev_to_bits(ds.out[0]), ref_out, "fused Hq=%d Hkv=%d d=%d part=%s" % (Hq, Hkv, d, partition))
+
+
+def test_decode_step_on_tiny_workload_and_with_poisoned_unused_slots():
+    h = wl.host_inputs(wl.workload("tiny"))
+    ref_pool, ref_out = oracle_step(h)
+    ds = run_step(h, fused=True)
+    assert np.array_equal(dev_to_bits(ds.pool.pool), ref_pool)
+    assert_close(dev_to_bits(ds.out[0]), ref_out, "tiny fused")
+    # the slot being appended to may hold anything before the step, NaN included
+    h = custom_inputs([5, 17, 70, 130, 1, 64, 33], 8, 2, 128, seed=19, extra_pages=2)
+    P = 16
+    live = np.zeros((h.num_pages, P), dtype=bool)
+    for r, L in enumerate(h.seq_lens.tolist()):
+        for j in range(L - 1):                                              # everything but the new token
+            live[h.block_tables[r, j // P], j % P] = True
+    pool = h.pool.reshape(1, h.num_pages, 2, 2, P, 128)
+    dead_pages, dead_slots = np.nonzero(~live)
+    pool[0, dead_pages, :, :, dead_slots, :] = 0x7FC0
+    ref_pool, ref_out = oracle_step(h)
+    assert np.all(np.isfinite(ref_out))
+    ds = run_step(h, fused=True)
+    assert np.array_equal(dev_to_bits(ds.pool.pool), ref_pool)
+    assert_close(dev_to_bits(ds.out[0]), ref_out, "fused, NaN in the target slots")
+
+
+def test_decode_step_reports_bad_append_pages_without_writing():
+    b = binding()
+    h = custom_inputs([50, 60], 8, 2, 128, seed=54)
+    h.block_tables[0, 3] = -7                                    # the append target of request 0
+    ds = make_device_step(h)
+    before = dev_to_bits(ds.pool.pool).copy()
+    ds.pool.decode_step(0, ds.bt, ds.sl, ds.q[0], ds.k_new[0], ds.v_new[0], ds.out[0])
+    assert ds.pool.check_status(raise_on_error=False) & b.STATUS_BAD_PAGE
+    after = dev_to_bits(ds.pool.pool).reshape(1, h.num_pages, 2, 2, 16, 128)
+    changed = (after != before.reshape(after.shape)).any(axis=-1)
+    assert int(changed.sum()) == 1 * 2 * 2                       # request 1 only
 
 
 # --------------------------------------------------------------------------- shapes and edges
@@ -213,30 +265,14 @@ def test_too_long_length_and_bad_page_id_are_reported_without_faulting():
 
 # --------------------------------------------------------------------------- the plan
 
-def expected_plan(lens_np, Hkv, C):
-    tiles = (lens_np.astype(np.int64) + 31) // 32
-    prefix = np.concatenate([[0], np.cumsum(tiles)]) * Hkv
-    total = int(prefix[-1])
-    q = max(1, -(-total // C))
-    starts = np.full((C, 4), -1, dtype=np.int32)
-    for c in range(C):
-        t0 = c * q
-        if t0 >= total:
-            continue
-        r = int(np.searchsorted(prefix, t0, side="right") - 1)
-        rem = t0 - int(prefix[r])
-        starts[c] = [r, rem // int(tiles[r]), rem % int(tiles[r]), t0]
-    return total, q, starts
-
-
 def check_plan(kp, lens_np, Hkv):
     sl = torch.from_numpy(lens_np).cuda()
     hdr, starts = kp.decode_plan(sl)
     C = kp.get_partition()
     total, q, want = expected_plan(lens_np, Hkv, C)
-    assert hdr["total_tiles"] == total and hdr["num_spans"] == C
-    assert hdr["tiles_per_span"] == q
-    assert hdr["spans_with_work"] == -(-total // q)
+    assert hdr["total_units"] == total and hdr["num_spans"] == C
+    assert hdr["units_per_span"] == q
+    assert hdr["spans_with_units"] == -(-total // q)
     assert np.array_equal(starts, want)
     return hdr
 
@@ -312,6 +348,35 @@ def full_parity(name, partitions=(None,)):
     return worst
 
 
+def full_parity_fused(name, partitions=(None,)):
+    w, lens, npg, bt, kp, pool_t, q, k, v, out = device_workload(name)
+    sh = pool_shape(w, npg)
+    host_pool = dev_to_bits(pool_t).reshape(-1)                  # state before the step
+    pristine = pool_t.clone()
+    hq, hk, hv = dev_to_bits(q), dev_to_bits(k), dev_to_bits(v)
+    assert oracle.kv_append(host_pool, sh, 0, bt, lens, hk[0], hv[0]) == 0
+    ref = oracle.decode_attention(host_pool, sh, 0, bt, lens, hq[0])
+    btd, sld = torch.from_numpy(bt).cuda(), torch.from_numpy(lens).cuda()
+    for part in partitions:
+        if part is not None:
+            kp.set_partition(part)
+        pool_t.copy_(pristine)                                   # every run appends into a pre-step pool
+        out.fill_(float("nan"))
+        kp.decode_step(0, btd, sld, q[0], k[0], v[0], out[0])
+        assert kp.check_status() == 0
+        assert np.array_equal(dev_to_bits(pool_t).reshape(-1), host_pool)
+        assert_close(dev_to_bits(out[0]), ref, "%s fused partition=%s" % (name, part))
+    kp.close()
+
+
+def test_llama8b_batch64_fused_step_full_parity():
+    full_parity_fused("llama8b_b64", partitions=(None, 100))
+
+
+def test_skewed_long_context_fused_step_full_parity():
+    full_parity_fused("skewed_long", partitions=(None, 2048))
+
+
 def test_llama8b_batch64_full_parity():
     full_parity("llama8b_b64", partitions=(None, 296, 100, 2048))
 
@@ -344,7 +409,7 @@ def test_step_latency_sweep_runs_nested_prefixes_and_counts_launches():
     med, mn = ds.pool.step_latency_sweep([1, 2, 4, 8], ds.bt, ds.sl, ds.q, ds.k_new, ds.v_new, ds.out,
                                          warmup=2, iters=5)
     assert med.shape == (4,) and np.all(med > 0) and np.all(mn > 0) and np.all(mn <= med)
-    assert ds.pool.launch_count() - n0 == 4 * (2 + 5) * 2 * 2    # sizes * steps * layers * kernels
+    assert ds.pool.launch_count() - n0 == 4 * (2 + 5) * 2 * 1    # sizes * steps * layers * one fused kernel
     # the last sweep point ran the full batch on both layers: outputs must be the oracle's
     sh = pool_shape(h.w, h.num_pages)
     ref_pool = h.pool.copy().reshape(-1)

@@ -20,6 +20,7 @@ constexpr int kTileTokens = kPageSize * kPagesPerTile;
 constexpr int kMaxGroup = 8;         // query heads per KV head handled by one MMA column block
 constexpr int kMaxSpans = 2048;      // upper bound on the partition width (one span per warp)
 constexpr int kMaxBatch = 8192;
+constexpr int kBulkMergeFrom = 4;    // merges of more partials than this go through shared memory
 
 constexpr uint32_t kStatusBadLength = 1u;
 constexpr uint32_t kStatusBadPage = 2u;
@@ -289,6 +290,20 @@ __device__ __forceinline__ void grid_launch_dependents()
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// 1-D bulk copy global -> shared, completion counted in bytes on an mbarrier (16-byte aligned, size % 16 == 0)
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ float4 ld_shared_f32x4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+
 __device__ __forceinline__ void fence_proxy_async()
 {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -477,6 +492,91 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
             *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
         }
     }
+}
+
+// The same merge for (request, kv head) pairs cut into many partials (small batches, very long
+// contexts): the partial accumulators are fetched with bulk async copies into the warp's ring --
+// idle once its span has been streamed -- up to `cap` partials per round, and summed from shared
+// memory.  A round costs one copy latency however many partials it holds.  `uses` counts how many
+// phases the mbarrier `bar` has completed so far and is advanced here.  Returns false if a
+// bounded wait gave up.
+template <int D>
+__device__ __noinline__ bool combine_partials_bulk(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
+                                                   uint16_t *out_rows, int s_first, int s_last, int slot_first, int G,
+                                                   int lane, uint32_t ring, int ring_bytes, uint32_t bar, int &uses,
+                                                   uint32_t *status)
+{
+    const int pieces = s_last - s_first + 1;
+    auto slot_of = [&](int i) { return i == 0 ? slot_first : 2 * (s_first + i); };
+    const int piece_bytes = G * D * 4;                       // the G live rows of a partial are contiguous
+    const int cap = min(32, ring_bytes / piece_bytes);
+
+    // running maximum over the rounds seen so far; sums are rescaled when it grows (online merge),
+    // so no separate pass over the (m, l) rows is needed
+    float mstar[kMaxGroup], lsum[kMaxGroup];
+    float4 acc[kMaxGroup];
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) { mstar[g] = -INFINITY; lsum[g] = 0.f; acc[g] = make_float4(0.f, 0.f, 0.f, 0.f); }
+    bool ok = true;
+    for (int base = 0; base < pieces && ok; base += cap) {
+        const int cnt = min(cap, pieces - base);
+        if (lane == 0) mbar_arrive_expect_tx(bar, cnt * piece_bytes);
+        __syncwarp();
+        float mi[kMaxGroup], li[kMaxGroup];
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g) { mi[g] = -INFINITY; li[g] = 0.f; }
+        if (lane < cnt) {                                     // lane i owns partial base + i of this round
+            const int slot = slot_of(base + lane);
+            bulk_load_1d(ring + lane * piece_bytes, part_acc + (size_t)slot * kMaxGroup * D, piece_bytes, bar);
+            const float *ml = part_ml + slot * 2 * kMaxGroup;
+            const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
+            const float4 c = ld_cg_f32x4(ml + 8), d = ld_cg_f32x4(ml + 12);
+            mi[0] = a.x; mi[1] = a.y; mi[2] = a.z; mi[3] = a.w; mi[4] = b.x; mi[5] = b.y; mi[6] = b.z; mi[7] = b.w;
+            li[0] = c.x; li[1] = c.y; li[2] = c.z; li[3] = c.w; li[4] = d.x; li[5] = d.y; li[6] = d.z; li[7] = d.w;
+        }
+        float f_mine[kMaxGroup];
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g) {
+            float mx = mi[g];
+#pragma unroll
+            for (int x = 16; x > 0; x >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, x));
+            const float mnew = fmaxf(mstar[g], mx);           // finite: every partial holds at least one token
+            const float rescale = fast_exp2(mstar[g] - mnew);
+            mstar[g] = mnew;
+            acc[g].x *= rescale; acc[g].y *= rescale; acc[g].z *= rescale; acc[g].w *= rescale;
+            f_mine[g] = fast_exp2(mi[g] - mnew);              // lanes without a partial: exp2(-inf) = 0
+            lsum[g] = lsum[g] * rescale + f_mine[g] * li[g];
+        }
+        ok = mbar_wait_bounded(bar, uses & 1, status);
+        ok = __all_sync(0xffffffffu, ok);
+        ++uses;
+        if (!ok) break;
+        for (int i = 0; i < cnt; ++i) {
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g) {
+                const float f = __shfl_sync(0xffffffffu, f_mine[g], i);
+                if (g < G && lane * 4 < D) {
+                    const float4 a = ld_shared_f32x4(ring + i * piece_bytes + g * D * 4 + lane * 16);
+                    acc[g].x += f * a.x; acc[g].y += f * a.y; acc[g].z += f * a.z; acc[g].w += f * a.w;
+                }
+            }
+        }
+        __syncwarp();                                         // all reads of this round precede the next round's copies
+    }
+    if (!ok) return false;
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) {
+#pragma unroll
+        for (int x = 16; x > 0; x >>= 1) lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], x);
+        if (g < G && lane * 4 < D) {
+            const float inv = 1.f / lsum[g];
+            uint2 packed;
+            packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
+            packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
+            *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
+        }
+    }
+    return true;
 }
 
 template <int D, int W, int NS>
@@ -944,8 +1044,20 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 if (last0) p.arrivals[pend_first[0]] = 0;
                 if (last1) p.arrivals[pend_first[1]] = 0;
             }
-            if (last0) combine_partials<D>(p.part_acc, p.part_ml, pend_out[0], pend_first[0], pend_last[0], pend_slot[0], G, lane);
-            if (last1) combine_partials<D>(p.part_acc, p.part_ml, pend_out[1], pend_first[1], pend_last[1], pend_slot[1], G, lane);
+            // stage 0's barrier has completed one phase per tile it carried; the ring is idle now
+            int bar_uses = (done + NS - 1) / NS;
+            fence_proxy_async();                  // partials written through the generic proxy, read by bulk copies
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                if (!(k == 0 ? last0 : last1)) continue;
+                const int pieces = pend_last[k] - pend_first[k] + 1;
+                if (alive && pieces > kBulkMergeFrom)
+                    alive = combine_partials_bulk<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k],
+                                                     pend_slot[k], G, lane, ring, NS * Lay::kStageBytes, bars, bar_uses,
+                                                     p.status);
+                else
+                    combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k], pend_slot[k], G, lane);
+            }
         }
     }
 
@@ -956,7 +1068,11 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     if (lane == 0) {
         p.trace[span * 8 + 3] = global_timer_ns();
         p.trace[span * 8 + 4] = t_wait;
+#ifdef CKV_TRACE_WAITS
         p.trace[span * 8 + 5] = t_between;
+#else
+        { unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); p.trace[span * 8 + 5] = smid; }
+#endif
 #ifdef CKV_TRACE_WAITS
         p.trace[span * 8 + 6] = t_issue;
         p.trace[span * 8 + 7] = t_masked;

@@ -494,6 +494,76 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
     }
 }
 
+// Merge of up to two (request, kv head) pairs with at most four partials each -- the usual case at
+// large batch, where a warp's first and last piece each pair up with a neighbour.  Lanes 0..3 own
+// the partials of pair 0, lanes 4..7 those of pair 1; every accumulator load of both pairs is
+// issued before any of them is needed, so the whole merge costs about one memory round trip.
+template <int D>
+__device__ __noinline__ void combine_small_pairs(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
+                                                 int n_pairs, int first0, int last0, int slot0, uint16_t *out0,
+                                                 int first1, int last1, int slot1, uint16_t *out1, int G, int lane)
+{
+    const int pair = (lane >> 2) & 1, pi = lane & 3;
+    const int my_first = pair ? first1 : first0, my_last = pair ? last1 : last0, my_slot0 = pair ? slot1 : slot0;
+    const bool mine = lane < 8 && pair < n_pairs && pi <= my_last - my_first;
+    float mi[kMaxGroup], li[kMaxGroup];
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) { mi[g] = -INFINITY; li[g] = 0.f; }
+    if (mine) {
+        const int slot = pi == 0 ? my_slot0 : 2 * (my_first + pi);
+        const float *ml = part_ml + slot * 2 * kMaxGroup;
+        const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
+        const float4 c = ld_cg_f32x4(ml + 8), d = ld_cg_f32x4(ml + 12);
+        mi[0] = a.x; mi[1] = a.y; mi[2] = a.z; mi[3] = a.w; mi[4] = b.x; mi[5] = b.y; mi[6] = b.z; mi[7] = b.w;
+        li[0] = c.x; li[1] = c.y; li[2] = c.z; li[3] = c.w; li[4] = d.x; li[5] = d.y; li[6] = d.z; li[7] = d.w;
+    }
+    float f_mine[kMaxGroup], lsum[kMaxGroup];
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) {                       // reductions stay inside each group of four lanes
+        float mx = fmaxf(mi[g], __shfl_xor_sync(0xffffffffu, mi[g], 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        f_mine[g] = mine ? fast_exp2(mi[g] - mx) : 0.f;
+        float ls = f_mine[g] * li[g];
+        ls += __shfl_xor_sync(0xffffffffu, ls, 1);
+        ls += __shfl_xor_sync(0xffffffffu, ls, 2);
+        lsum[g] = ls;
+    }
+#pragma unroll
+    for (int it = 0; it < 2; ++it) {
+        if (it >= n_pairs) break;
+        const int f0 = it ? first1 : first0, pieces = (it ? last1 : last0) - f0 + 1, s0 = it ? slot1 : slot0;
+        uint16_t *out_rows = it ? out1 : out0;
+        float4 acc[kMaxGroup];
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (i >= pieces) break;
+            const int slot = i == 0 ? s0 : 2 * (f0 + i);
+            const float *pa = part_acc + (size_t)slot * kMaxGroup * D + lane * 4;
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g) {
+                const float f = __shfl_sync(0xffffffffu, f_mine[g], it * 4 + i);
+                if (g < G && lane * 4 < D) {
+                    const float4 a = ld_cg_f32x4(pa + g * D);
+                    acc[g].x += f * a.x; acc[g].y += f * a.y; acc[g].z += f * a.z; acc[g].w += f * a.w;
+                }
+            }
+        }
+#pragma unroll
+        for (int g = 0; g < kMaxGroup; ++g) {
+            const float lg = __shfl_sync(0xffffffffu, lsum[g], it * 4);
+            if (g < G && lane * 4 < D) {
+                const float inv = 1.f / lg;
+                uint2 packed;
+                packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
+                packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
+                *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
+            }
+        }
+    }
+}
+
 // The same merge for (request, kv head) pairs cut into many partials (small batches, very long
 // contexts): the partial accumulators are fetched with bulk async copies into the warp's ring --
 // idle once its span has been streamed -- up to `cap` partials per round, and summed from shared
@@ -1044,19 +1114,30 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 if (last0) p.arrivals[pend_first[0]] = 0;
                 if (last1) p.arrivals[pend_first[1]] = 0;
             }
-            // stage 0's barrier has completed one phase per tile it carried; the ring is idle now
-            int bar_uses = (done + NS - 1) / NS;
-            fence_proxy_async();                  // partials written through the generic proxy, read by bulk copies
+            const int pieces0 = last0 ? pend_last[0] - pend_first[0] + 1 : 0;
+            const int pieces1 = last1 ? pend_last[1] - pend_first[1] + 1 : 0;
+            if (pieces0 <= kBulkMergeFrom && pieces1 <= kBulkMergeFrom) {
+                // the usual case: one or two short merges, done together
+                const int a = last0 ? 0 : 1, b = 1;
+                combine_small_pairs<D>(p.part_acc, p.part_ml, (last0 ? 1 : 0) + (last1 ? 1 : 0),
+                                       pend_first[a], pend_last[a], pend_slot[a], pend_out[a],
+                                       pend_first[b], pend_last[b], pend_slot[b], pend_out[b], G, lane);
+            } else {
+                // stage 0's barrier has completed one phase per tile it carried; the ring is idle now
+                int bar_uses = (done + NS - 1) / NS;
+                fence_proxy_async();              // partials written through the generic proxy, read by bulk copies
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                if (!(k == 0 ? last0 : last1)) continue;
-                const int pieces = pend_last[k] - pend_first[k] + 1;
-                if (alive && pieces > kBulkMergeFrom)
-                    alive = combine_partials_bulk<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k],
-                                                     pend_slot[k], G, lane, ring, NS * Lay::kStageBytes, bars, bar_uses,
-                                                     p.status);
-                else
-                    combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k], pend_slot[k], G, lane);
+                for (int k = 0; k < 2; ++k) {
+                    if (!(k == 0 ? last0 : last1)) continue;
+                    const int pieces = pend_last[k] - pend_first[k] + 1;
+                    if (alive && pieces > kBulkMergeFrom)
+                        alive = combine_partials_bulk<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k],
+                                                         pend_slot[k], G, lane, ring, NS * Lay::kStageBytes, bars,
+                                                         bar_uses, p.status);
+                    else
+                        combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k],
+                                            pend_slot[k], G, lane);
+                }
             }
         }
     }

@@ -38,6 +38,10 @@ METRIC = "decode_attention_hbm_bandwidth"
 UNIT = "TB/s"
 NORMALISED_TO_TBS = 8.0          # the metric is quoted as a fraction of 8 TB/s
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on the headline
+# workload, from the ncu capture summarised in profiles/paged_decode_attn_llama8b_b64.md.  Set to
+# None whenever the kernel changes after the capture.
+NCU_TRAFFIC_BYTES = 576.8e6
 
 
 # ------------------------------------------------------------------------------- clocks
@@ -340,7 +344,7 @@ def run_ours(args) -> None:
     achieved = attn_bytes / (attn_ms / attn_n * 1e-3) / 1e9
     roofline = {"bound": "hbm", "kernel": "paged_decode_attn_kernel (fused append + plan + attention + combine)", "achieved": achieved, "peak": peak,
                 "unit": "GB/s", "frac": achieved / peak, "peak_kind": "of " + peak_kind,
-                "traffic": None, "bytes_per_launch": attn_bytes, "us_per_launch": attn_ms / attn_n * 1e3,
+                "traffic": NCU_TRAFFIC_BYTES, "bytes_per_launch": attn_bytes, "us_per_launch": attn_ms / attn_n * 1e3,
                 "frac_of_8TBs": achieved / (NORMALISED_TO_TBS * 1e3)}
 
     # ---- end to end through the host-buffer entry point (pinned memory, copies inside the timing)

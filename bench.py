@@ -386,6 +386,7 @@ def run_ours(args) -> None:
     if rank == 0 and world == 1:
         if not args.no_sweep:
             line["latency_sweep"] = run_sweep(dev)
+            line["local_autoscaler"] = run_autoscaler(line["latency_sweep"])
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(HEADLINE)
     if rank == 0:
@@ -411,6 +412,24 @@ def run_sweep(dev) -> dict:
                      "tokens_per_s": round(b / (m * 1e-6)), "tbs": round(nb / (m * 1e-6) / 1e12, 3)})
     dw.kp.close()
     return {"workload": "mixed_sweep", "l2": "256 MB flush before every timed step", "points": rows}
+
+
+def run_autoscaler(sweep: dict) -> dict:
+    """Algorithm 1 closed over the measured curve: ITL(batch) = layers x attention(batch) + a constant
+    standing for weight streaming, against the paper's interactive (200 ms) and batch (2 s) ITL SLOs."""
+    from paper_2501_08090_b200 import binding
+    sizes = [p["batch"] for p in sweep["points"]]
+    layers, weights_us = 32, 2300.0          # Llama-3-8B: 32 layers; ~16 GB of bf16 weights at ~7 TB/s
+    us = [layers * p["us_per_step"] for p in sweep["points"]]
+    out = {"model": "ITL = 32 layers x measured attention step + 2.3 ms weight streaming", "alpha": 0.5, "runs": []}
+    for slo_ms in (200.0, 2000.0):
+        max_bs, batch, itl, bp = binding.autoscaler_simulate(slo_ms * 1e3, 8.0, sizes, us, weights_us,
+                                                             demand=1 << 20, iterations=400, max_bs=65536.0)
+        tail = batch[200:]
+        out["runs"].append({"itl_slo_ms": slo_ms, "peak_batch": int(tail.max()), "trough_batch": int(tail.min()),
+                            "max_itl_ms": round(float(itl[200:].max()) / 1e3, 2),
+                            "updates_to_first_halving": int(np.argmax(bp >= 1.0)) if (bp >= 1.0).any() else None})
+    return out
 
 
 def main() -> None:

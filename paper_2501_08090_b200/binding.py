@@ -26,6 +26,8 @@ EXPORTS = (
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
     "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace", "ckv_set_overlap",
     "decode_attention_noalloc", "decode_step",
+    "local_autoscaler_instance_slo", "local_autoscaler_create", "local_autoscaler_destroy",
+    "local_autoscaler_update", "local_autoscaler_get", "local_autoscaler_simulate",
 )
 
 
@@ -33,6 +35,11 @@ class CkvError(RuntimeError):
     def __init__(self, code: int, message: str):
         super().__init__("chiron_kv error %d: %s" % (code, message))
         self.code = code
+
+
+class AutoscalerConfig(ctypes.Structure):
+    _fields_ = [("alpha", ctypes.c_double), ("itl_slo_us", ctypes.c_double),
+                ("min_bs", ctypes.c_double), ("max_bs", ctypes.c_double)]
 
 
 class Config(ctypes.Structure):
@@ -71,6 +78,15 @@ def _load() -> ctypes.CDLL:
     lib.ckv_read_span_trace.restype = i32; lib.ckv_read_span_trace.argtypes = [vp, vp, vp, vp]
     lib.decode_attention_noalloc.restype = i32
     lib.decode_attention_noalloc.argtypes = [cfgp, vp, i32, i32, vp, vp, vp, vp, i32, vp, ctypes.POINTER(ctypes.c_uint32)]
+    f64 = ctypes.c_double
+    f64p, i32p, acfgp = ctypes.POINTER(f64), ctypes.POINTER(i32), ctypes.POINTER(AutoscalerConfig)
+    lib.local_autoscaler_instance_slo.restype = i32; lib.local_autoscaler_instance_slo.argtypes = [vp, i32, f64p]
+    lib.local_autoscaler_create.restype = i32; lib.local_autoscaler_create.argtypes = [acfgp, f64, ctypes.POINTER(vp)]
+    lib.local_autoscaler_destroy.restype = i32; lib.local_autoscaler_destroy.argtypes = [vp]
+    lib.local_autoscaler_update.restype = i32; lib.local_autoscaler_update.argtypes = [vp, f64, f64, f64p, f64p]
+    lib.local_autoscaler_get.restype = i32; lib.local_autoscaler_get.argtypes = [vp, f64p]
+    lib.local_autoscaler_simulate.restype = i32
+    lib.local_autoscaler_simulate.argtypes = [acfgp, f64, i32, vp, vp, f64, i32, i32, vp, vp, vp, vp]
     lib.ckv_launch_count.restype = i64; lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_last_error.restype = ctypes.c_char_p; lib.ckv_last_error.argtypes = []
     return lib
@@ -268,3 +284,65 @@ def decode_attention_noalloc(cfg: Config, pool: torch.Tensor, layer: int, block_
                                       _stream_ptr(stream), ctypes.byref(bits) if sync else None)
     _check(rc)
     return int(bits.value)
+
+
+class LocalAutoscaler:
+    """Per-instance batch-size autoscaler (Algorithm 1); host-only, thin wrapper over the C ABI."""
+
+    def __init__(self, itl_slo_us: float, initial_max_bs: float, alpha: float = 0.5,
+                 min_bs: float = 1.0, max_bs: float = 1e9):
+        self.cfg = AutoscalerConfig(alpha, itl_slo_us, min_bs, max_bs)
+        self._h = ctypes.c_void_p()
+        rc = lib.local_autoscaler_create(ctypes.byref(self.cfg), float(initial_max_bs), ctypes.byref(self._h))
+        if rc != CKV_OK:
+            raise CkvError(rc, "local_autoscaler_create: bad configuration")
+
+    def update(self, itl_us: float, throughput: float):
+        """(new maximum batch size, backpressure)."""
+        bs, bp = ctypes.c_double(0.0), ctypes.c_double(0.0)
+        rc = lib.local_autoscaler_update(self._h, float(itl_us), float(throughput), ctypes.byref(bs), ctypes.byref(bp))
+        if rc != CKV_OK:
+            raise CkvError(rc, "local_autoscaler_update: bad argument")
+        return bs.value, bp.value
+
+    @property
+    def max_bs(self) -> float:
+        v = ctypes.c_double(0.0)
+        lib.local_autoscaler_get(self._h, ctypes.byref(v))
+        return v.value
+
+    def close(self):
+        if self._h.value:
+            lib.local_autoscaler_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def instance_slo(itl_slos_us) -> float:
+    a = np.ascontiguousarray(itl_slos_us, dtype=np.float64)
+    out = ctypes.c_double(0.0)
+    rc = lib.local_autoscaler_instance_slo(a.ctypes.data, int(a.size), ctypes.byref(out))
+    if rc != CKV_OK:
+        raise CkvError(rc, "local_autoscaler_instance_slo: bad argument")
+    return out.value
+
+
+def autoscaler_simulate(itl_slo_us: float, initial_max_bs: float, batch_sizes, us_per_step, extra_us: float,
+                        demand: int, iterations: int, alpha: float = 0.5, min_bs: float = 1.0, max_bs: float = 1e9):
+    """Closed loop of Algorithm 1 over a latency curve: arrays (MaxBS, batch run, ITL us, backpressure)."""
+    cfg = AutoscalerConfig(alpha, itl_slo_us, min_bs, max_bs)
+    x = np.ascontiguousarray(batch_sizes, dtype=np.float64)
+    y = np.ascontiguousarray(us_per_step, dtype=np.float64)
+    o_bs = np.zeros(iterations, np.float64); o_b = np.zeros(iterations, np.int32)
+    o_itl = np.zeros(iterations, np.float64); o_bp = np.zeros(iterations, np.float64)
+    rc = lib.local_autoscaler_simulate(ctypes.byref(cfg), float(initial_max_bs), int(x.size), x.ctypes.data,
+                                       y.ctypes.data, float(extra_us), int(demand), int(iterations),
+                                       o_bs.ctypes.data, o_b.ctypes.data, o_itl.ctypes.data, o_bp.ctypes.data)
+    if rc != CKV_OK:
+        raise CkvError(rc, "local_autoscaler_simulate: bad argument")
+    return o_bs, o_b, o_itl, o_bp

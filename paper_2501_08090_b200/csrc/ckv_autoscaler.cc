@@ -1,0 +1,136 @@
+// Local batch-size autoscaler (include/chiron_autoscaler.h): Algorithm 1 of the paper and a
+// closed-loop driver over a measured latency curve.  Host-only.
+#include "chiron_autoscaler.h"
+
+#include <algorithm>
+#include <cmath>
+#include <limits>
+#include <new>
+
+namespace {
+constexpr int32_t kOk = 0, kInval = -1, kNoMem = -2;
+
+bool config_ok(const ckv_autoscaler_config *c)
+{
+    return c && c->alpha > 0.0 && c->alpha <= 1.0 && c->itl_slo_us > 0.0 && c->min_bs >= 1.0 && c->max_bs >= c->min_bs;
+}
+
+double clamp(double x, double lo, double hi) { return std::min(std::max(x, lo), hi); }
+}  // namespace
+
+struct ckv_autoscaler {
+    ckv_autoscaler_config cfg;
+    double max_bs;
+    double prev_throughput;
+    bool has_prev;
+};
+
+namespace {
+double step(ckv_autoscaler &a, double itl_us, double throughput, double *bp_out)
+{
+    const double lbp = itl_us / a.cfg.itl_slo_us;
+    double tbp = 0.0;
+    if (a.has_prev) tbp = throughput > 0.0 ? a.prev_throughput / throughput : std::numeric_limits<double>::infinity();
+    const double bp = std::max(lbp, tbp);
+    double next;
+    if (bp < 1.0)
+        next = bp > 0.0 ? a.cfg.alpha * (1.0 / bp) * a.max_bs + (1.0 - a.cfg.alpha) * a.max_bs : a.cfg.max_bs;
+    else
+        next = a.max_bs / 2.0;
+    next = clamp(next, a.cfg.min_bs, a.cfg.max_bs);
+    // TBP asks whether the last INCREASE of the batch size paid off: keep the baseline only across one
+    a.has_prev = next > a.max_bs;
+    a.prev_throughput = throughput;
+    a.max_bs = next;
+    if (bp_out) *bp_out = bp;
+    return a.max_bs;
+}
+
+double curve(int32_t n, const double *x, const double *y, double bs)
+{
+    if (n == 1 || bs <= x[0]) return y[0];
+    int i = 1;
+    while (i < n - 1 && bs > x[i]) ++i;
+    return y[i - 1] + (y[i] - y[i - 1]) * (bs - x[i - 1]) / (x[i] - x[i - 1]);
+}
+}  // namespace
+
+extern "C" {
+
+int32_t local_autoscaler_instance_slo(const double *itl_slos_us, int32_t n, double *out_slo_us)
+{
+    if (!itl_slos_us || n < 1 || !out_slo_us) return kInval;
+    double m = itl_slos_us[0];
+    for (int32_t i = 1; i < n; ++i) m = std::min(m, itl_slos_us[i]);
+    if (!(m > 0.0)) return kInval;
+    *out_slo_us = m;
+    return kOk;
+}
+
+int32_t local_autoscaler_create(const ckv_autoscaler_config *cfg, double initial_max_bs, ckv_autoscaler **out)
+{
+    if (!out) return kInval;
+    *out = nullptr;
+    if (!config_ok(cfg) || !(initial_max_bs >= 1.0)) return kInval;
+    ckv_autoscaler *a = new (std::nothrow) ckv_autoscaler();
+    if (!a) return kNoMem;
+    a->cfg = *cfg;
+    a->max_bs = clamp(initial_max_bs, cfg->min_bs, cfg->max_bs);
+    a->prev_throughput = 0.0;
+    a->has_prev = false;
+    *out = a;
+    return kOk;
+}
+
+int32_t local_autoscaler_destroy(ckv_autoscaler *a)
+{
+    if (!a) return kInval;
+    delete a;
+    return kOk;
+}
+
+int32_t local_autoscaler_update(ckv_autoscaler *a, double itl_us, double throughput, double *out_max_bs,
+                                double *out_backpressure)
+{
+    if (!a || !out_max_bs || !(itl_us > 0.0) || std::isnan(throughput)) return kInval;
+    *out_max_bs = step(*a, itl_us, throughput, out_backpressure);
+    return kOk;
+}
+
+int32_t local_autoscaler_get(const ckv_autoscaler *a, double *out_max_bs)
+{
+    if (!a || !out_max_bs) return kInval;
+    *out_max_bs = a->max_bs;
+    return kOk;
+}
+
+int32_t local_autoscaler_simulate(const ckv_autoscaler_config *cfg, double initial_max_bs, int32_t n_points,
+                                  const double *batch_sizes, const double *us_per_step, double extra_us,
+                                  int32_t demand, int32_t iterations, double *out_max_bs, int32_t *out_batch,
+                                  double *out_itl_us, double *out_backpressure)
+{
+    if (!config_ok(cfg) || !(initial_max_bs >= 1.0) || n_points < 1 || !batch_sizes || !us_per_step) return kInval;
+    if (demand < 1 || iterations < 1 || extra_us < 0.0) return kInval;
+    for (int32_t i = 0; i < n_points; ++i) {
+        if (!(us_per_step[i] > 0.0) || !(batch_sizes[i] >= 1.0)) return kInval;
+        if (i > 0 && !(batch_sizes[i] > batch_sizes[i - 1])) return kInval;
+    }
+    ckv_autoscaler a;
+    a.cfg = *cfg;
+    a.max_bs = clamp(initial_max_bs, cfg->min_bs, cfg->max_bs);
+    a.prev_throughput = 0.0;
+    a.has_prev = false;
+    for (int32_t k = 0; k < iterations; ++k) {
+        const int32_t bs = std::max<int32_t>(1, (int32_t)std::min<double>(std::floor(a.max_bs), (double)demand));
+        const double itl = curve(n_points, batch_sizes, us_per_step, (double)bs) + extra_us;
+        double bp = 0.0;
+        const double next = step(a, itl, (double)bs / itl, &bp);
+        if (out_max_bs) out_max_bs[k] = next;
+        if (out_batch) out_batch[k] = bs;
+        if (out_itl_us) out_itl_us[k] = itl;
+        if (out_backpressure) out_backpressure[k] = bp;
+    }
+    return kOk;
+}
+
+}  // extern "C"

@@ -387,6 +387,7 @@ def run_ours(args) -> None:
         if not args.no_sweep:
             line["latency_sweep"] = run_sweep(dev)
             line["local_autoscaler"] = run_autoscaler(line["latency_sweep"])
+            line["kv_swap"] = run_swap(dev)
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(HEADLINE)
     if rank == 0:
@@ -412,6 +413,38 @@ def run_sweep(dev) -> dict:
                      "tokens_per_s": round(b / (m * 1e-6)), "tbs": round(nb / (m * 1e-6) / 1e12, 3)})
     dw.kp.close()
     return {"workload": "mixed_sweep", "l2": "256 MB flush before every timed step", "points": rows}
+
+
+def run_swap(dev) -> dict:
+    """Swap-out / swap-in of a 4096-page request image (8B shape, one layer: 256 MB) through the
+    library's zero-copy kernels, beside torch's pinned-memory copies of the same bytes."""
+    import torch
+    from paper_2501_08090_b200 import binding
+    n_pages, total_pages = 4096, 8192
+    cfg = binding.make_config(1, 32, 8, 128, total_pages, n_pages, 1)
+    kp = binding.KvPool(cfg, device=dev)
+    kp.pool.normal_()
+    ids = torch.randperm(total_pages, device=dev)[:n_pages].to(torch.int32)
+    nbytes = kp.swap_image_bytes(n_pages)
+    image = torch.empty(nbytes // 2, dtype=torch.int16).pin_memory()
+    dev_buf = torch.empty(nbytes // 2, dtype=torch.int16, device=dev)
+
+    def timed(fn, reps=5):
+        fn(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record(); torch.cuda.synchronize()
+        return nbytes * reps / (e0.elapsed_time(e1) * 1e-3) / 1e9
+    out = {"bytes": nbytes, "pages": n_pages,
+           "swap_out_gbs": round(timed(lambda: kp.swap_out(ids, image)), 2),
+           "swap_in_gbs": round(timed(lambda: kp.swap_in(ids, image)), 2),
+           "memcpy_d2h_gbs": round(timed(lambda: image.copy_(dev_buf, non_blocking=True)), 2),
+           "memcpy_h2d_gbs": round(timed(lambda: dev_buf.copy_(image, non_blocking=True)), 2)}
+    kp.check_status()
+    kp.close()
+    return out
 
 
 def run_autoscaler(sweep: dict) -> dict:

@@ -221,6 +221,27 @@ int32_t ckv_read_span_trace(ckv_pool *pool, void *stream, uint64_t *h_trace, int
 int64_t ckv_launch_count(const ckv_pool *pool);
 
 /*
+ * KV swap-out / swap-in: move one request's pages, for every layer, between the pool and a
+ * contiguous image in host memory (Section 3 "Request Multiplexing with Mixed Instances": an
+ * interactive request may evict a batch request from a mixed instance, and the evicted request's
+ * KV cache is saved by migrating it to CPU memory so that it can restart fast).
+ *   d_page_ids  int32 [n_pages] on the device: the request's block-table row (physical page ids,
+ *               in context order).  For swap-in these may be different pages than at swap-out.
+ *   h_image     PINNED host memory (cudaHostAlloc / cudaHostRegister, 16-byte aligned) the device
+ *               can address; the kernels read and write it directly, there is no staging copy.
+ *               Layout: bf16 [num_layers][n_pages][num_kv_heads][2][page_size][head_dim];
+ *               image_bytes >= num_layers * n_pages * (bytes of one page in one layer).
+ * Both calls only enqueue one kernel on `stream`; the image is complete (swap-out) or reusable
+ * (swap-in) once the stream has reached that point.  A page id outside the pool is skipped and
+ * flagged in the status word.  Bit-exact.
+ * Errors: CKV_EINVAL (arguments, unpinned image), CKV_ENOMEM (image too small), CKV_ECUDA.
+ */
+int32_t kv_swap_out(ckv_pool *pool, int32_t n_pages, const int32_t *d_page_ids, void *h_image,
+                    size_t image_bytes, void *stream);
+int32_t kv_swap_in(ckv_pool *pool, int32_t n_pages, const int32_t *d_page_ids, const void *h_image,
+                   size_t image_bytes, void *stream);
+
+/*
  * decode_attention without a workspace.  (The paper has no counterpart; this entry point exists
  * for integration reasons only.)
  *

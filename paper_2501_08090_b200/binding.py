@@ -25,7 +25,7 @@ EXPORTS = (
     "decode_attention", "decode_plan", "ckv_set_partition", "ckv_get_partition", "kv_check_status",
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
     "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace", "ckv_set_overlap",
-    "decode_attention_noalloc", "decode_step",
+    "decode_attention_noalloc", "decode_step", "kv_swap_out", "kv_swap_in",
     "local_autoscaler_instance_slo", "local_autoscaler_create", "local_autoscaler_destroy",
     "local_autoscaler_update", "local_autoscaler_get", "local_autoscaler_simulate",
 )
@@ -64,6 +64,8 @@ def _load() -> ctypes.CDLL:
     lib.kv_append.restype = i32; lib.kv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.decode_attention.restype = i32; lib.decode_attention.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     lib.decode_step.restype = i32; lib.decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
+    lib.kv_swap_out.restype = i32; lib.kv_swap_out.argtypes = [vp, i32, vp, vp, sz, vp]
+    lib.kv_swap_in.restype = i32; lib.kv_swap_in.argtypes = [vp, i32, vp, vp, sz, vp]
     lib.decode_plan.restype = i32; lib.decode_plan.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_set_partition.restype = i32; lib.ckv_set_partition.argtypes = [vp, i32]
     lib.ckv_set_overlap.restype = i32; lib.ckv_set_overlap.argtypes = [vp, i32]
@@ -195,6 +197,24 @@ class KvPool:
                                _dev_ptr(seq_lens, torch.int32), _dev_ptr(q, torch.bfloat16),
                                _dev_ptr(k_new, torch.bfloat16), _dev_ptr(v_new, torch.bfloat16),
                                _dev_ptr(out, torch.bfloat16), _stream_ptr(stream)))
+
+    def swap_image_bytes(self, n_pages: int) -> int:
+        c = self.cfg
+        return c.num_layers * int(n_pages) * c.num_kv_heads * 2 * c.page_size * c.head_dim * 2
+
+    def swap_out(self, page_ids, image, stream=None) -> None:
+        """Copy the listed pages (all layers) into `image`, a pinned host tensor."""
+        self._swap(lib.kv_swap_out, page_ids, image, stream)
+
+    def swap_in(self, page_ids, image, stream=None) -> None:
+        """Copy `image` (pinned host tensor) into the listed pages (all layers)."""
+        self._swap(lib.kv_swap_in, page_ids, image, stream)
+
+    def _swap(self, fn, page_ids, image, stream):
+        if image.is_cuda or not image.is_contiguous() or not image.is_pinned():
+            raise ValueError("the swap image must be a contiguous pinned host tensor")
+        _check(fn(self._h, int(page_ids.shape[0]), _dev_ptr(page_ids, torch.int32), image.data_ptr(),
+                  image.numel() * image.element_size(), _stream_ptr(stream)))
 
     def decode_plan(self, seq_lens, stream=None):
         """(header dict, int32 [num_spans][4] array of span starts)."""

@@ -698,4 +698,53 @@ int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int3
     return CKV_OK;
 }
 
+static int32_t swap_launch(ckv_pool *pool, const char *fn, bool to_host, int32_t n_pages, const int32_t *d_page_ids,
+                           void *h_image, size_t image_bytes, void *stream)
+{
+    if (!pool) return fail(CKV_EINVAL, "%s: pool is NULL", fn);
+    if (n_pages < 1 || !d_page_ids || !h_image) return fail(CKV_EINVAL, "%s: bad page list or image", fn);
+    const ckv_config &c = pool->cfg;
+    const size_t page_bytes = (size_t)c.num_kv_heads * 2 * c.page_size * c.head_dim * 2;
+    const size_t need = (size_t)c.num_layers * n_pages * page_bytes;
+    if (image_bytes < need) return fail(CKV_ENOMEM, "%s: image holds %zu bytes, %zu needed", fn, image_bytes, need);
+    if (reinterpret_cast<uintptr_t>(h_image) & 15u) return fail(CKV_EINVAL, "%s: image not 16-byte aligned", fn);
+    void *d_image = nullptr;
+    cudaError_t e = cudaHostGetDevicePointer(&d_image, h_image, 0);
+    if (e != cudaSuccess || !d_image) {
+        cudaGetLastError();
+        return fail(CKV_EINVAL, "%s: the image must be pinned host memory the device can address (%s)", fn,
+                    cudaGetErrorString(e));
+    }
+    ckv::SwapParams sp{};
+    sp.pool = reinterpret_cast<uint4 *>(pool->d_pool);
+    sp.image = static_cast<uint4 *>(d_image);
+    sp.page_ids = d_page_ids;
+    sp.status = pool->wsp<uint32_t>(pool->ws.status);
+    sp.n_pages = n_pages;
+    sp.num_layers = c.num_layers;
+    sp.num_pages = c.num_pages;
+    sp.page_vecs = (int32_t)(page_bytes / 16);
+    const long long work = (long long)need / 16;
+    const int threads = 256;
+    const int blocks = (int)std::min<long long>((work + threads - 1) / threads, (long long)pool->num_sms * 8);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (to_host) ckv::kv_swap_kernel<true><<<blocks, threads, 0, s>>>(sp);
+    else ckv::kv_swap_kernel<false><<<blocks, threads, 0, s>>>(sp);
+    CKV_CUDA(cudaGetLastError());
+    pool->launches += 1;
+    return CKV_OK;
+}
+
+int32_t kv_swap_out(ckv_pool *pool, int32_t n_pages, const int32_t *d_page_ids, void *h_image, size_t image_bytes,
+                    void *stream)
+{
+    return swap_launch(pool, "kv_swap_out", true, n_pages, d_page_ids, h_image, image_bytes, stream);
+}
+
+int32_t kv_swap_in(ckv_pool *pool, int32_t n_pages, const int32_t *d_page_ids, const void *h_image,
+                   size_t image_bytes, void *stream)
+{
+    return swap_launch(pool, "kv_swap_in", false, n_pages, d_page_ids, const_cast<void *>(h_image), image_bytes, stream);
+}
+
 }  // extern "C"

@@ -102,6 +102,41 @@ __global__ void kv_append_kernel(const AppendParams p)
 }
 
 // ------------------------------------------------------------------------------------------
+// KV swap: one request's pages, all layers, between the pool and a contiguous image in pinned host
+// memory that the device reaches directly (no staging copy).  One thread moves 16 bytes at a time.
+// Image layout: [layer][i][kv_head][K|V][slot][d], i = position in page_ids.
+// ------------------------------------------------------------------------------------------
+struct SwapParams {
+    uint4 *pool;                    // whole pool
+    uint4 *image;                   // device-visible address of the host image
+    const int32_t *page_ids;        // [n_pages]
+    uint32_t *status;
+    int32_t n_pages, num_layers, num_pages;
+    int32_t page_vecs;              // 16-byte pieces per (layer, page): Hkv*2*16*d*2/16
+};
+
+template <bool kToHost>
+__global__ void kv_swap_kernel(const SwapParams p)
+{
+    const long long per_layer = (long long)p.n_pages * p.page_vecs;
+    const long long total = per_layer * p.num_layers;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int layer = (int)(idx / per_layer);
+        const long long rem = idx % per_layer;
+        const int i = (int)(rem / p.page_vecs), v = (int)(rem % p.page_vecs);
+        const int page = __ldg(p.page_ids + i);
+        if (page < 0 || page >= p.num_pages) {
+            if (v == 0 && layer == 0) atomicOr(p.status, kStatusBadPage);
+            continue;
+        }
+        uint4 *in_pool = p.pool + ((size_t)layer * p.num_pages + page) * p.page_vecs + v;
+        if (kToHost) p.image[idx] = *in_pool;
+        else *in_pool = p.image[idx];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // K2: the split-KV plan.
 //
 // The attention kernel derives its partition from seq_lens in its own prologue (warp_plan below),

@@ -472,7 +472,7 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
     float mstar[kMaxGroup];
 #pragma unroll
     for (int g = 0; g < kMaxGroup; ++g) mstar[g] = -INFINITY;
-    for (int base = (pieces - 1) & ~31; base >= 0; base -= 32) {       // round 0 last: its values stay in mi, li
+    for (int base = (pieces - 1) & ~31; base >= 0; base -= 32) {       // chunk 0 last: its values stay in mi, li
         if (base + lane < pieces) {
             load_ml(base + lane);
 #pragma unroll

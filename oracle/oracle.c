@@ -274,3 +274,111 @@ int32_t oracle_decode_attention(const uint16_t *pool, int32_t num_layers, int32_
     }
     return rc;
 }
+
+/*
+ * Multi-token step (speculative-decoding verification, chunked append: paper Section 4 lists
+ * speculative decoding and chunked prefill among the optimizations an instance may run with;
+ * Section 6 "Experiment Setup" evaluates with speculative decoding enabled).  Each request appends
+ * q_len tokens in this iteration: positions L_r - q_len .. L_r - 1 (seq_lens again hold the length
+ * AFTER the append).  New token i's key/value rows go to page block_tables[r][pos / P], slot
+ * pos % P, pos = L_r - q_len + i.
+ *   k_new, v_new  bf16 bits [batch][q_len][num_kv_heads][head_dim]
+ * Returns 0; -1 bad length (L < q_len or beyond the table); -4 page id out of range.
+ */
+int32_t oracle_kv_append_multi(uint16_t *pool, int32_t num_layers, int32_t num_pages,
+                               int32_t num_kv_heads, int32_t page_size, int32_t head_dim,
+                               int32_t layer, int32_t batch, int32_t q_len, int32_t max_pages_per_req,
+                               const int32_t *block_tables, const int32_t *seq_lens,
+                               const uint16_t *k_new, const uint16_t *v_new)
+{
+    if (layer < 0 || layer >= num_layers || q_len < 1) return -1;
+    int32_t rc = 0;
+    for (int32_t r = 0; r < batch; ++r) {
+        int32_t L = seq_lens[r];
+        if (L < q_len || (int64_t)L > (int64_t)max_pages_per_req * page_size) { rc = -1; continue; }
+        for (int32_t i = 0; i < q_len; ++i) {
+            int32_t pos = L - q_len + i;
+            int32_t page = block_tables[(size_t)r * max_pages_per_req + pos / page_size];
+            int32_t slot = pos % page_size;
+            if (page < 0 || page >= num_pages) { rc = -4; continue; }
+            for (int32_t kh = 0; kh < num_kv_heads; ++kh) {
+                size_t src = (((size_t)r * q_len + i) * num_kv_heads + kh) * (size_t)head_dim;
+                size_t dk = pool_row_offset(num_pages, num_kv_heads, page_size, head_dim, layer, page, kh, 0, slot);
+                size_t dv = pool_row_offset(num_pages, num_kv_heads, page_size, head_dim, layer, page, kh, 1, slot);
+                for (int32_t c = 0; c < head_dim; ++c) {
+                    pool[dk + c] = k_new[src + c];
+                    pool[dv + c] = v_new[src + c];
+                }
+            }
+        }
+    }
+    return rc;
+}
+
+/*
+ * Causal attention of the q_len new tokens of every request: query token i (position
+ * L_r - q_len + i) attends to tokens 0 .. L_r - q_len + i, i.e. to everything before it and to
+ * itself, through the dense definition above.
+ *   q    bf16 bits [batch][q_len][num_q_heads][head_dim]
+ *   out  fp64      [batch][q_len][num_q_heads][head_dim]
+ * Returns 0; -1 bad length; -4 page id out of range.
+ */
+int32_t oracle_decode_attention_multi(const uint16_t *pool, int32_t num_layers, int32_t num_pages,
+                                      int32_t num_q_heads, int32_t num_kv_heads, int32_t page_size,
+                                      int32_t head_dim, int32_t layer, int32_t batch, int32_t q_len,
+                                      int32_t max_pages_per_req, const int32_t *block_tables,
+                                      const int32_t *seq_lens, const uint16_t *q, double *out)
+{
+    if (layer < 0 || layer >= num_layers || q_len < 1) return -1;
+    if (num_kv_heads < 1 || num_q_heads % num_kv_heads != 0) return -1;
+    const int32_t G = num_q_heads / num_kv_heads;
+    const int32_t d = head_dim;
+    const double scale = 1.0 / sqrt((double)d);
+    int32_t rc = 0;
+    for (int32_t r = 0; r < batch; ++r) {
+        int32_t L = seq_lens[r];
+        if (L < q_len || (int64_t)L > (int64_t)max_pages_per_req * page_size) return -1;
+        int32_t np = (L + page_size - 1) / page_size;
+        for (int32_t i = 0; i < np; ++i) {
+            int32_t page = block_tables[(size_t)r * max_pages_per_req + i];
+            if (page < 0 || page >= num_pages) return -4;
+        }
+    }
+    const int64_t npairs = (int64_t)batch * num_kv_heads;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t pair = 0; pair < npairs; ++pair) {
+        const int32_t r = (int32_t)(pair / num_kv_heads);
+        const int32_t kh = (int32_t)(pair % num_kv_heads);
+        const int64_t L = seq_lens[r];
+        double *K = (double *)malloc((size_t)L * d * sizeof(double));
+        double *V = (double *)malloc((size_t)L * d * sizeof(double));
+        double *qd = (double *)malloc((size_t)d * sizeof(double));
+        if (!K || !V || !qd) {
+#pragma omp atomic write
+            rc = -2;
+            free(K); free(V); free(qd);
+            continue;
+        }
+        for (int64_t j = 0; j < L; ++j) {
+            int32_t page = block_tables[(size_t)r * max_pages_per_req + j / page_size];
+            int32_t slot = (int32_t)(j % page_size);
+            size_t ok = pool_row_offset(num_pages, num_kv_heads, page_size, d, layer, page, kh, 0, slot);
+            size_t ov = pool_row_offset(num_pages, num_kv_heads, page_size, d, layer, page, kh, 1, slot);
+            for (int32_t c = 0; c < d; ++c) {
+                K[j * d + c] = bf16_bits_to_f64(pool[ok + c]);
+                V[j * d + c] = bf16_bits_to_f64(pool[ov + c]);
+            }
+        }
+        for (int32_t i = 0; i < q_len; ++i) {
+            const int64_t visible = L - q_len + 1 + i;          /* tokens 0 .. own position */
+            for (int32_t g = 0; g < G; ++g) {
+                const int32_t h = kh * G + g;
+                const size_t qo = (((size_t)r * q_len + i) * num_q_heads + h) * (size_t)d;
+                for (int32_t c = 0; c < d; ++c) qd[c] = bf16_bits_to_f64(q[qo + c]);
+                oracle_attention_dense_f64(qd, K, V, visible, d, scale, out + qo, NULL);
+            }
+        }
+        free(K); free(V); free(qd);
+    }
+    return rc;
+}

@@ -35,6 +35,11 @@ def _load():
         lib.oracle_decode_attention.restype = i32
         lib.oracle_decode_attention.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, i32,
                                                 vp, vp, vp, vp]
+        lib.oracle_kv_append_multi.restype = i32
+        lib.oracle_kv_append_multi.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+        lib.oracle_decode_attention_multi.restype = i32
+        lib.oracle_decode_attention_multi.argtypes = [vp, i32, i32, i32, i32, i32, i32, i32, i32, i32, i32,
+                                                      vp, vp, vp, vp]
         _lib = lib
     return _lib
 
@@ -123,4 +128,33 @@ def decode_attention(pool: np.ndarray, shape: PoolShape, layer: int, block_table
                                          _p(bt), _p(sl), _p(qq), _p(out))
     if rc != 0:
         raise ValueError("oracle_decode_attention failed: %d" % rc)
+    return out
+
+
+def kv_append_multi(pool: np.ndarray, shape: PoolShape, layer: int, q_len: int, block_tables, seq_lens,
+                    k_new, v_new) -> int:
+    """In-place append of q_len new tokens per request (k_new, v_new [batch][q_len][Hkv][d])."""
+    assert pool.dtype == np.uint16 and pool.flags.c_contiguous and pool.size == shape.elems
+    bt = _c(block_tables, np.int32); sl = _c(seq_lens, np.int32)
+    k = _c(k_new, np.uint16); v = _c(v_new, np.uint16)
+    batch, max_pages = bt.shape
+    assert k.size == batch * q_len * shape.num_kv_heads * shape.head_dim == v.size
+    return int(_load().oracle_kv_append_multi(_p(pool), shape.num_layers, shape.num_pages, shape.num_kv_heads,
+                                              shape.page_size, shape.head_dim, layer, batch, q_len, max_pages,
+                                              _p(bt), _p(sl), _p(k), _p(v)))
+
+
+def decode_attention_multi(pool: np.ndarray, shape: PoolShape, layer: int, q_len: int, block_tables, seq_lens,
+                           q) -> np.ndarray:
+    """Causal attention of the q_len new tokens: fp64 [batch][q_len][Hq][d]."""
+    assert pool.dtype == np.uint16 and pool.flags.c_contiguous and pool.size == shape.elems
+    bt = _c(block_tables, np.int32); sl = _c(seq_lens, np.int32); qq = _c(q, np.uint16)
+    batch, max_pages = bt.shape
+    assert qq.size == batch * q_len * shape.num_q_heads * shape.head_dim
+    out = np.zeros((batch, q_len, shape.num_q_heads, shape.head_dim), dtype=np.float64)
+    rc = _load().oracle_decode_attention_multi(_p(pool), shape.num_layers, shape.num_pages, shape.num_q_heads,
+                                               shape.num_kv_heads, shape.page_size, shape.head_dim, layer, batch,
+                                               q_len, max_pages, _p(bt), _p(sl), _p(qq), _p(out))
+    if rc != 0:
+        raise ValueError("oracle_decode_attention_multi failed: %d" % rc)
     return out

@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on the headline
 # workload, from the ncu capture summarised in profiles/paged_decode_attn_llama8b_b64.md.  Set to
 # None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES = 576.8e6
+NCU_TRAFFIC_BYTES = None      # kernel changed since the last capture (576.8 MB then)
 
 
 # ------------------------------------------------------------------------------- clocks
@@ -388,6 +388,7 @@ def run_ours(args) -> None:
             line["latency_sweep"] = run_sweep(dev)
             line["local_autoscaler"] = run_autoscaler(line["latency_sweep"])
             line["kv_swap"] = run_swap(dev)
+            line["multi_token_step"] = run_multi_token(dw)
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(HEADLINE)
     if rank == 0:
@@ -445,6 +446,35 @@ def run_swap(dev) -> dict:
     kp.check_status()
     kp.close()
     return out
+
+
+def run_multi_token(dw) -> dict:
+    """kv_append_multi + decode_attention_multi on the headline batch: q_len new tokens per request
+    share one pass over the KV stream (q_len x group <= 8 columns)."""
+    import torch
+    w, rows = dw.w, []
+    for q_len in range(1, 8 // w.group + 1):
+        q = wl.device_normal_bf16((dw.B, q_len, w.num_q_heads, w.head_dim), w.seed, 20 + q_len, dw.device)
+        k = wl.device_normal_bf16((dw.B, q_len, w.num_kv_heads, w.head_dim), w.seed, 30 + q_len, dw.device)
+        out = torch.zeros_like(q)
+
+        def step():
+            dw.kp.kv_append_multi(0, q_len, dw.bt, dw.sl, k, k)
+            dw.kp.decode_attention_multi(0, q_len, dw.bt, dw.sl, q, out)
+        for _ in range(5):
+            step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n = 200
+        e0.record()
+        for _ in range(n):
+            step()
+        e1.record(); torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) * 1e3 / n
+        rows.append({"q_len": q_len, "us_per_step": round(us, 2), "kv_tbs": round(dw.bytes["kv"] / us / 1e6, 3),
+                     "new_tokens_per_s": round(dw.B * q_len / us * 1e6)})
+    dw.kp.check_status()
+    return {"workload": dw.w.name, "launches_per_step": 2, "points": rows}
 
 
 def run_autoscaler(sweep: dict) -> dict:

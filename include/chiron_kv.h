@@ -131,6 +131,29 @@ int32_t decode_step(ckv_pool *pool, int32_t layer, int32_t batch,
                     void *stream);
 
 /*
+ * Multi-token step: every request appends q_len tokens in this iteration and the q_len new tokens
+ * attend causally -- new token i (position seq_lens[r] - q_len + i) sees the context up to and
+ * including itself.  This is the verification pass of speculative decoding and a chunk of chunked
+ * prefill, which the paper lists among the optimizations an instance may run with (Section 4,
+ * "Why use an online algorithm?"; Section 6 "Experiment Setup").  seq_lens hold the lengths AFTER
+ * the q_len tokens are appended; requests with seq_lens[r] < q_len are unusable (status bit, rows
+ * zero-filled).
+ *   kv_append_multi         d_k_new, d_v_new: bf16 [batch][q_len][num_kv_heads][head_dim]; 1 <= q_len <= 8
+ *   decode_attention_multi  d_q, d_out: bf16 [batch][q_len][num_q_heads][head_dim]; the new tokens'
+ *                           queries share the 8 columns of one tensor-core pass with the heads of
+ *                           the group, so the KV stream is read once for all of them; this needs
+ *                           q_len * (num_q_heads / num_kv_heads) <= 8, otherwise CKV_EINVAL.
+ * Call kv_append_multi first: attention reads the new tokens' keys and values from the pool.
+ * Errors: CKV_EINVAL, CKV_ECUDA.
+ */
+int32_t kv_append_multi(ckv_pool *pool, int32_t layer, int32_t batch, int32_t q_len,
+                        const int32_t *d_block_tables, const int32_t *d_seq_lens,
+                        const void *d_k_new, const void *d_v_new, void *stream);
+int32_t decode_attention_multi(ckv_pool *pool, int32_t layer, int32_t batch, int32_t q_len,
+                               const int32_t *d_block_tables, const int32_t *d_seq_lens,
+                               const void *d_q, void *d_out, void *stream);
+
+/*
  * The split-KV partition decode_attention uses for these lengths, copied to the host for
  * inspection (runs a small kernel and synchronises `stream`; decode_attention itself derives the
  * same partition inside its attention kernel and launches no plan kernel).  A "tile" is 32

@@ -26,6 +26,7 @@ EXPORTS = (
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
     "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace", "ckv_set_overlap",
     "decode_attention_noalloc", "decode_step", "kv_swap_out", "kv_swap_in",
+    "kv_append_multi", "decode_attention_multi",
     "local_autoscaler_instance_slo", "local_autoscaler_create", "local_autoscaler_destroy",
     "local_autoscaler_update", "local_autoscaler_get", "local_autoscaler_simulate",
 )
@@ -66,6 +67,8 @@ def _load() -> ctypes.CDLL:
     lib.decode_step.restype = i32; lib.decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.kv_swap_out.restype = i32; lib.kv_swap_out.argtypes = [vp, i32, vp, vp, sz, vp]
     lib.kv_swap_in.restype = i32; lib.kv_swap_in.argtypes = [vp, i32, vp, vp, sz, vp]
+    lib.kv_append_multi.restype = i32; lib.kv_append_multi.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.decode_attention_multi.restype = i32; lib.decode_attention_multi.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.decode_plan.restype = i32; lib.decode_plan.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_set_partition.restype = i32; lib.ckv_set_partition.argtypes = [vp, i32]
     lib.ckv_set_overlap.restype = i32; lib.ckv_set_overlap.argtypes = [vp, i32]
@@ -197,6 +200,18 @@ class KvPool:
                                _dev_ptr(seq_lens, torch.int32), _dev_ptr(q, torch.bfloat16),
                                _dev_ptr(k_new, torch.bfloat16), _dev_ptr(v_new, torch.bfloat16),
                                _dev_ptr(out, torch.bfloat16), _stream_ptr(stream)))
+
+    def kv_append_multi(self, layer: int, q_len: int, block_tables, seq_lens, k_new, v_new, stream=None) -> None:
+        """Append q_len new tokens per request (k_new, v_new [batch][q_len][Hkv][d])."""
+        _check(lib.kv_append_multi(self._h, layer, int(seq_lens.shape[0]), int(q_len),
+                                   _dev_ptr(block_tables, torch.int32), _dev_ptr(seq_lens, torch.int32),
+                                   _dev_ptr(k_new, torch.bfloat16), _dev_ptr(v_new, torch.bfloat16), _stream_ptr(stream)))
+
+    def decode_attention_multi(self, layer: int, q_len: int, block_tables, seq_lens, q, out, stream=None) -> None:
+        """Causal attention of the q_len new tokens (q, out [batch][q_len][Hq][d])."""
+        _check(lib.decode_attention_multi(self._h, layer, int(seq_lens.shape[0]), int(q_len),
+                                          _dev_ptr(block_tables, torch.int32), _dev_ptr(seq_lens, torch.int32),
+                                          _dev_ptr(q, torch.bfloat16), _dev_ptr(out, torch.bfloat16), _stream_ptr(stream)))
 
     def swap_image_bytes(self, n_pages: int) -> int:
         c = self.cfg

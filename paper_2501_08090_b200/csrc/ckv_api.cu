@@ -336,12 +336,14 @@ int32_t ckv_set_overlap(ckv_pool *pool, int32_t enable)
 
 int64_t ckv_launch_count(const ckv_pool *pool) { return pool ? pool->launches : 0; }
 
-int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
-                  const int32_t *d_seq_lens, const void *d_k_new, const void *d_v_new, void *stream)
+static int32_t append_launch(ckv_pool *pool, const char *fn, int32_t layer, int32_t batch, int32_t q_len,
+                             const int32_t *d_block_tables, const int32_t *d_seq_lens, const void *d_k_new,
+                             const void *d_v_new, void *stream)
 {
-    if (int32_t rc = check_call(pool, layer, batch, "kv_append")) return rc;
-    if (!d_block_tables || !d_seq_lens || !d_k_new || !d_v_new) return fail(CKV_EINVAL, "kv_append: NULL argument");
-    if (!aligned16(d_k_new) || !aligned16(d_v_new)) return fail(CKV_EINVAL, "kv_append: k_new/v_new not 16-byte aligned");
+    if (int32_t rc = check_call(pool, layer, batch, fn)) return rc;
+    if (q_len < 1 || q_len > ckv::kMaxGroup) return fail(CKV_EINVAL, "%s: q_len %d outside [1, 8]", fn, q_len);
+    if (!d_block_tables || !d_seq_lens || !d_k_new || !d_v_new) return fail(CKV_EINVAL, "%s: NULL argument", fn);
+    if (!aligned16(d_k_new) || !aligned16(d_v_new)) return fail(CKV_EINVAL, "%s: k_new/v_new not 16-byte aligned", fn);
     const ckv_config &c = pool->cfg;
     ckv::AppendParams ap{};
     const size_t layer_bytes = (size_t)c.num_pages * c.num_kv_heads * 2 * c.page_size * c.head_dim * 2;
@@ -356,7 +358,8 @@ int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d
     ap.num_pages = c.num_pages;
     ap.num_kv_heads = c.num_kv_heads;
     ap.head_dim = c.head_dim;
-    const long long work = (long long)batch * c.num_kv_heads * 2 * (c.head_dim / 8);
+    ap.q_len = q_len;
+    const long long work = (long long)batch * q_len * c.num_kv_heads * 2 * (c.head_dim / 8);
     const int threads = 256;
     const int blocks = (int)std::min<long long>((work + threads - 1) / threads, 4096);
     cudaLaunchConfig_t lc{};
@@ -373,12 +376,29 @@ int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d
     return CKV_OK;
 }
 
+int32_t kv_append(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
+                  const int32_t *d_seq_lens, const void *d_k_new, const void *d_v_new, void *stream)
+{
+    return append_launch(pool, "kv_append", layer, batch, 1, d_block_tables, d_seq_lens, d_k_new, d_v_new, stream);
+}
+
+int32_t kv_append_multi(ckv_pool *pool, int32_t layer, int32_t batch, int32_t q_len, const int32_t *d_block_tables,
+                        const int32_t *d_seq_lens, const void *d_k_new, const void *d_v_new, void *stream)
+{
+    return append_launch(pool, "kv_append_multi", layer, batch, q_len, d_block_tables, d_seq_lens, d_k_new, d_v_new,
+                         stream);
+}
+
 // Attention for one layer, optionally with the KV append folded into the same kernel.
-static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, int32_t batch,
+static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, int32_t batch, int32_t q_len,
                                 const int32_t *d_block_tables, const int32_t *d_seq_lens, const void *d_q,
                                 const void *d_k_new, const void *d_v_new, void *d_out, void *stream)
 {
     if (int32_t rc = check_call(pool, layer, batch, fn)) return rc;
+    if (q_len < 1 || q_len * (pool->cfg.num_q_heads / pool->cfg.num_kv_heads) > ckv::kMaxGroup)
+        return fail(CKV_EINVAL, "%s: q_len %d x group %d exceeds the %d columns one pass holds", fn, q_len,
+                    pool->cfg.num_q_heads / pool->cfg.num_kv_heads, ckv::kMaxGroup);
+    if (q_len > 1 && d_k_new) return fail(CKV_EINVAL, "%s: the fused append is for single-token steps", fn);
     if (!d_block_tables || !d_seq_lens || !d_q || !d_out) return fail(CKV_EINVAL, "%s: NULL argument", fn);
     if (!aligned16(d_q) || !aligned16(d_out)) return fail(CKV_EINVAL, "%s: q/out not 16-byte aligned", fn);
     if ((d_k_new == nullptr) != (d_v_new == nullptr)) return fail(CKV_EINVAL, "%s: k_new and v_new go together", fn);
@@ -409,6 +429,7 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
     ap.group = c.num_q_heads / c.num_kv_heads;
     ap.layer_page_base = layer * c.num_pages;
     ap.num_spans = pool->num_spans;
+    ap.q_len = q_len;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
 
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -437,8 +458,16 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
 int32_t decode_attention(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
                          const int32_t *d_seq_lens, const void *d_q, void *d_out, void *stream)
 {
-    return attention_launch(pool, "decode_attention", layer, batch, d_block_tables, d_seq_lens, d_q, nullptr, nullptr,
-                            d_out, stream);
+    return attention_launch(pool, "decode_attention", layer, batch, 1, d_block_tables, d_seq_lens, d_q, nullptr,
+                            nullptr, d_out, stream);
+}
+
+int32_t decode_attention_multi(ckv_pool *pool, int32_t layer, int32_t batch, int32_t q_len,
+                               const int32_t *d_block_tables, const int32_t *d_seq_lens, const void *d_q,
+                               void *d_out, void *stream)
+{
+    return attention_launch(pool, "decode_attention_multi", layer, batch, q_len, d_block_tables, d_seq_lens, d_q,
+                            nullptr, nullptr, d_out, stream);
 }
 
 int32_t decode_step(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
@@ -446,7 +475,7 @@ int32_t decode_step(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t 
                     void *d_out, void *stream)
 {
     if (!d_k_new || !d_v_new) return fail(CKV_EINVAL, "decode_step: NULL k_new/v_new");
-    return attention_launch(pool, "decode_step", layer, batch, d_block_tables, d_seq_lens, d_q, d_k_new, d_v_new,
+    return attention_launch(pool, "decode_step", layer, batch, 1, d_block_tables, d_seq_lens, d_q, d_k_new, d_v_new,
                             d_out, stream);
 }
 
@@ -682,6 +711,7 @@ int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int3
     ap.group = cfg->num_q_heads / cfg->num_kv_heads;
     ap.layer_page_base = layer * cfg->num_pages;
     ap.num_spans = num_spans;
+    ap.q_len = 1;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)cfg->head_dim));
 
     int32_t rc;

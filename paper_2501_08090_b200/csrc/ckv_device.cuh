@@ -45,10 +45,11 @@ struct PlanHeader {
     int32_t spans_with_units;
 };
 
-// A context length is usable if 1 <= L <= table capacity; otherwise the request has no tiles.
-__host__ __device__ __forceinline__ int tiles_of_length(int L, int max_pages_per_req)
+// A context length is usable if min_len <= L <= table capacity (min_len = the number of new
+// tokens of the step, 1 for plain decode); otherwise the request has no tiles.
+__host__ __device__ __forceinline__ int tiles_of_length(int L, int max_pages_per_req, int min_len = 1)
 {
-    if (L < 1 || (long long)L > (long long)max_pages_per_req * kPageSize) return 0;
+    if (L < min_len || (long long)L > (long long)max_pages_per_req * kPageSize) return 0;
     return (L + kTileTokens - 1) / kTileTokens;
 }
 
@@ -63,6 +64,7 @@ struct AppendParams {
     const uint4 *v_new;
     uint32_t *status;
     int32_t batch, max_pages_per_req, num_pages, num_kv_heads, head_dim;
+    int32_t q_len;                  // new tokens per request: k_new, v_new are [batch][q_len][Hkv][d]
 };
 
 __global__ void kv_append_kernel(const AppendParams p)
@@ -72,30 +74,33 @@ __global__ void kv_append_kernel(const AppendParams p)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int vec_per_row = p.head_dim / 8;                       // 16-byte pieces per row
-    const int per_req = p.num_kv_heads * 2 * vec_per_row;
+    const int per_tok = p.num_kv_heads * 2 * vec_per_row;
+    const int per_req = per_tok * p.q_len;
     const long long total = (long long)p.batch * per_req;
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
         const int r = (int)(idx / per_req);
         int rem = (int)(idx % per_req);
+        const int qi = rem / per_tok;                                 // which of the request's new tokens
+        rem -= qi * per_tok;
         const int kh = rem / (2 * vec_per_row);
         rem -= kh * 2 * vec_per_row;
         const int kv = rem / vec_per_row;
         const int c = rem % vec_per_row;
 
         const int L = p.seq_lens[r];
-        if (tiles_of_length(L, p.max_pages_per_req) == 0) {
+        if (tiles_of_length(L, p.max_pages_per_req, p.q_len) == 0) {
             if (rem == 0 && kh == 0) atomicOr(p.status, kStatusBadLength);
             continue;
         }
-        const int pos = L - 1;
+        const int pos = L - p.q_len + qi;
         const int page = p.block_tables[(size_t)r * p.max_pages_per_req + pos / kPageSize];
         if (page < 0 || page >= p.num_pages) {
             if (rem == 0 && kh == 0) atomicOr(p.status, kStatusBadPage);
             continue;
         }
         const int slot = pos % kPageSize;
-        const uint4 *src = (kv == 0 ? p.k_new : p.v_new) + ((size_t)r * p.num_kv_heads + kh) * vec_per_row + c;
+        const uint4 *src = (kv == 0 ? p.k_new : p.v_new) + (((size_t)r * p.q_len + qi) * p.num_kv_heads + kh) * vec_per_row + c;
         const size_t row = (((size_t)page * p.num_kv_heads + kh) * 2 + kv) * kPageSize + slot;
         p.pool_layer[row * vec_per_row + c] = *src;
     }
@@ -155,12 +160,12 @@ struct SpanStart {
 // Requests with an unusable length get their output rows cleared and the status word flagged.
 // Executed by one warp of the grid.
 __device__ __forceinline__ void flag_unusable_requests(const int32_t *__restrict__ seq_lens, int batch,
-                                                       int max_pages_per_req, int lane, uint16_t *out,
+                                                       int max_pages_per_req, int min_len, int lane, uint16_t *out,
                                                        int out_row_elems, uint32_t *status)
 {
     for (int base = 0; base < batch; base += 32) {
         const int r = base + lane;
-        const bool bad = r < batch && tiles_of_length(__ldg(seq_lens + r), max_pages_per_req) == 0;
+        const bool bad = r < batch && tiles_of_length(__ldg(seq_lens + r), max_pages_per_req, min_len) == 0;
         unsigned todo = __ballot_sync(0xffffffffu, bad);
         if (todo && lane == 0) atomicOr(status, kStatusBadLength);
         while (todo) {                                   // the whole warp clears one row at a time
@@ -178,13 +183,13 @@ __device__ __forceinline__ int units_of_tiles(int t) { return t > 0 ? t + kPiece
 // Executed by one whole warp.  Two passes over seq_lens: the total number of units, then the
 // (request, kv head) that holds unit span*q and the first tile at or after it.
 __device__ __forceinline__ SpanStart warp_plan(const int32_t *__restrict__ seq_lens, int batch, int max_pages_per_req,
-                                               int num_kv_heads, int num_spans, int span, int lane)
+                                               int num_kv_heads, int num_spans, int span, int lane, int min_len = 1)
 {
     SpanStart s;
     int sum = 0;
     for (int base = 0; base < batch; base += 32) {
         const int r = base + lane;
-        if (r < batch) sum += units_of_tiles(tiles_of_length(__ldg(seq_lens + r), max_pages_per_req));
+        if (r < batch) sum += units_of_tiles(tiles_of_length(__ldg(seq_lens + r), max_pages_per_req, min_len));
     }
 #pragma unroll
     for (int x = 16; x > 0; x >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, x);
@@ -200,7 +205,7 @@ __device__ __forceinline__ SpanStart warp_plan(const int32_t *__restrict__ seq_l
     for (int base = 0; base < batch; base += 32) {
         const int r = base + lane;
         const int L = r < batch ? __ldg(seq_lens + r) : 0;
-        const int t = r < batch ? tiles_of_length(L, max_pages_per_req) : 0;
+        const int t = r < batch ? tiles_of_length(L, max_pages_per_req, min_len) : 0;
         int incl = units_of_tiles(t);
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -446,16 +451,22 @@ struct AttnParams {
     int32_t batch, max_pages_per_req, num_pages, num_kv_heads, num_q_heads, group;
     int32_t layer_page_base;        // layer * num_pages
     int32_t num_spans;
+    int32_t q_len;                  // new tokens per request in this step (1 for plain decode); q_len*group <= 8
     float scale_log2;               // log2(e) / sqrt(d)
 };
 
+// Columns.  The 8 columns of the MMA hold (new token, head of the group) pairs: column c is new
+// token c / G and head c % G, ncols = q_len * G <= 8 of them are live.  With one new token per
+// request (the usual decode step) a column is simply a head.  Output rows of a (request, kv head)
+// start at out_rows; column c's row is out_rows + (c / G) * qi_stride + (c % G) * D.
+//
 // Merge the partials of one (request, kv head) that spans s_first..s_last hold, and write its bf16
 // output rows.  Run by one whole warp (the last one to arrive for that pair).  Loads are issued in
 // batches so the merge costs a few L2 round trips, not one per partial.
 template <int D>
 __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
-                                              uint16_t *out_rows, int s_first, int s_last, int slot_first, int G,
-                                              int lane)
+                                              uint16_t *out_rows, int s_first, int s_last, int slot_first, int ncols, int G,
+                                              int qi_stride, int lane)
 {
     const int pieces = s_last - s_first + 1;
     auto slot_of = [&](int i) { return i == 0 ? slot_first : 2 * (s_first + i); };
@@ -508,7 +519,7 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
 #pragma unroll
             for (int g = 0; g < kMaxGroup; ++g) {
                 const float f = __shfl_sync(0xffffffffu, f_mine[g], i);
-                if (g < G && lane * 4 < D) {
+                if (g < ncols && lane * 4 < D) {
                     const float4 a = ld_cg_f32x4(pa + g * D);
                     acc[g].x += f * a.x; acc[g].y += f * a.y; acc[g].z += f * a.z; acc[g].w += f * a.w;
                 }
@@ -519,12 +530,12 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
     for (int g = 0; g < kMaxGroup; ++g) {
 #pragma unroll
         for (int x = 16; x > 0; x >>= 1) lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], x);
-        if (g < G && lane * 4 < D) {
+        if (g < ncols && lane * 4 < D) {
             const float inv = 1.f / lsum[g];
             uint2 packed;
             packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
             packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
-            *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
+            *(uint2 *)(out_rows + (size_t)(g / G) * qi_stride + (size_t)(g % G) * D + lane * 4) = packed;
         }
     }
 }
@@ -536,7 +547,8 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
 template <int D>
 __device__ __noinline__ void combine_small_pairs(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
                                                  int n_pairs, int first0, int last0, int slot0, uint16_t *out0,
-                                                 int first1, int last1, int slot1, uint16_t *out1, int G, int lane)
+                                                 int first1, int last1, int slot1, uint16_t *out1, int ncols, int G,
+                                                 int qi_stride, int lane)
 {
     const int pair = (lane >> 2) & 1, pi = lane & 3;
     const int my_first = pair ? first1 : first0, my_last = pair ? last1 : last0, my_slot0 = pair ? slot1 : slot0;
@@ -579,7 +591,7 @@ __device__ __noinline__ void combine_small_pairs(const float *__restrict__ part_
 #pragma unroll
             for (int g = 0; g < kMaxGroup; ++g) {
                 const float f = __shfl_sync(0xffffffffu, f_mine[g], it * 4 + i);
-                if (g < G && lane * 4 < D) {
+                if (g < ncols && lane * 4 < D) {
                     const float4 a = ld_cg_f32x4(pa + g * D);
                     acc[g].x += f * a.x; acc[g].y += f * a.y; acc[g].z += f * a.z; acc[g].w += f * a.w;
                 }
@@ -588,12 +600,12 @@ __device__ __noinline__ void combine_small_pairs(const float *__restrict__ part_
 #pragma unroll
         for (int g = 0; g < kMaxGroup; ++g) {
             const float lg = __shfl_sync(0xffffffffu, lsum[g], it * 4);
-            if (g < G && lane * 4 < D) {
+            if (g < ncols && lane * 4 < D) {
                 const float inv = 1.f / lg;
                 uint2 packed;
                 packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
                 packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
-                *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
+                *(uint2 *)(out_rows + (size_t)(g / G) * qi_stride + (size_t)(g % G) * D + lane * 4) = packed;
             }
         }
     }
@@ -607,13 +619,13 @@ __device__ __noinline__ void combine_small_pairs(const float *__restrict__ part_
 // bounded wait gave up.
 template <int D>
 __device__ __noinline__ bool combine_partials_bulk(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
-                                                   uint16_t *out_rows, int s_first, int s_last, int slot_first, int G,
-                                                   int lane, uint32_t ring, int ring_bytes, uint32_t bar, int &uses,
+                                                   uint16_t *out_rows, int s_first, int s_last, int slot_first, int ncols,
+                                                   int G, int qi_stride, int lane, uint32_t ring, int ring_bytes, uint32_t bar, int &uses,
                                                    uint32_t *status)
 {
     const int pieces = s_last - s_first + 1;
     auto slot_of = [&](int i) { return i == 0 ? slot_first : 2 * (s_first + i); };
-    const int piece_bytes = G * D * 4;                       // the G live rows of a partial are contiguous
+    const int piece_bytes = ncols * D * 4;                   // the live rows of a partial are contiguous
     const int cap = min(32, ring_bytes / piece_bytes);
 
     // running maximum over the rounds seen so far; sums are rescaled when it grows (online merge),
@@ -660,7 +672,7 @@ __device__ __noinline__ bool combine_partials_bulk(const float *__restrict__ par
 #pragma unroll
             for (int g = 0; g < kMaxGroup; ++g) {
                 const float f = __shfl_sync(0xffffffffu, f_mine[g], i);
-                if (g < G && lane * 4 < D) {
+                if (g < ncols && lane * 4 < D) {
                     const float4 a = ld_shared_f32x4(ring + i * piece_bytes + g * D * 4 + lane * 16);
                     acc[g].x += f * a.x; acc[g].y += f * a.y; acc[g].z += f * a.z; acc[g].w += f * a.w;
                 }
@@ -673,12 +685,12 @@ __device__ __noinline__ bool combine_partials_bulk(const float *__restrict__ par
     for (int g = 0; g < kMaxGroup; ++g) {
 #pragma unroll
         for (int x = 16; x > 0; x >>= 1) lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], x);
-        if (g < G && lane * 4 < D) {
+        if (g < ncols && lane * 4 < D) {
             const float inv = 1.f / lsum[g];
             uint2 packed;
             packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
             packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
-            *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
+            *(uint2 *)(out_rows + (size_t)(g / G) * qi_stride + (size_t)(g % G) * D + lane * 4) = packed;
         }
     }
     return true;
@@ -717,7 +729,7 @@ struct SpanCursor {
         do {
             if (++r >= p.batch) return false;
             L = __ldg(p.seq_lens + r);
-            tiles = tiles_of_length(L, p.max_pages_per_req);
+            tiles = tiles_of_length(L, p.max_pages_per_req, p.q_len);
         } while (tiles == 0);
         return true;
     }
@@ -751,10 +763,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     // ---- plan: where does this warp's span start?
     // Nothing read up to the dependency wait below is written by the preceding kernel of a decode
     // step (the KV append writes only the pool), so this prologue overlaps that kernel's tail.
-    const SpanStart st = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane);
+    const SpanStart st = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane,
+                                   p.q_len);
     if (st.r < 0 || span == 0) {
         grid_dependency_wait();
-        if (span == 0) flag_unusable_requests(p.seq_lens, p.batch, p.max_pages_per_req, lane, p.out, p.num_q_heads * D, p.status);
+        if (span == 0)
+            flag_unusable_requests(p.seq_lens, p.batch, p.max_pages_per_req, p.q_len, lane, p.out,
+                                   p.q_len * p.num_q_heads * D, p.status);
     }
     if (st.r < 0) {
         if (lane == 0) {
@@ -768,6 +783,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     const long long v_end = st.end;
     const int q_span = st.q;
     const int G = p.group;
+    const int ncols = G * p.q_len;               // live MMA columns: column c = new token c / G, head c % G
+    const int qi_stride = p.num_q_heads * D;     // elements between a request's consecutive new tokens in q / out
 
     // ---- issue side: block-table entries travel in registers, 32 pages (16 tiles) per chunk
     SpanCursor ic;
@@ -791,13 +808,14 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     // query fragments of a (request, kv head), fetched when the issue cursor enters it
     uint32_t qn[Lay::kKSteps][2];
     int qn_r = -1, qn_h = -1;
-    const int g_row = lane >> 2;                 // query head (within the group) this lane loads Q for
+    const int c_row = lane >> 2;                 // the column this lane loads Q for
     auto load_q = [&](uint32_t (&dst)[Lay::kKSteps][2], int r, int h) {
-        const uint32_t *qrow = (const uint32_t *)(p.q + ((size_t)r * p.num_q_heads + h * G + g_row) * D);
+        const uint32_t *qrow = (const uint32_t *)(p.q + ((size_t)r * p.q_len + c_row / G) * qi_stride +
+                                                  (size_t)(h * G + c_row % G) * D);
 #pragma unroll
         for (int ks = 0; ks < Lay::kKSteps; ++ks) {
-            dst[ks][0] = g_row < G ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
-            dst[ks][1] = g_row < G ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
+            dst[ks][0] = c_row < ncols ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
+            dst[ks][1] = c_row < ncols ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
         }
     };
 
@@ -944,8 +962,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             ++landed;
             if (done == 0 && lane == 0) p.trace[span * 8 + 1] = global_timer_ns();
 
-            const int ntok = min(kTileTokens, piece_L - ti * kTileTokens);      // valid tokens in this tile
-            const bool full_tile = (ntok == kTileTokens);
+            const int ntok = min(kTileTokens, piece_L - ti * kTileTokens);      // tokens of the context in this tile
+            // Causality among the step's new tokens: column c (new token c / G) sees the context up to
+            // and including its own position, i.e. vis_all + c / G tokens; every column sees vis_all.
+            const int vis_all = piece_L - p.q_len + 1;
+            const bool full_tile = (ti + 1) * kTileTokens <= vis_all;
+            const int lim0 = min(ntok, vis_all + g0 / G - ti * kTileTokens);         // visible tokens of this tile,
+            const int lim1 = min(ntok, vis_all + (g0 + 1) / G - ti * kTileTokens);   // for this lane's two columns
             const int np = (ntok + kPageSize - 1) / kPageSize;
             const uint32_t sb = ring + slot * Lay::kStageBytes;
 
@@ -1016,7 +1039,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int tok = mt * kPageSize + (lane >> 2) + (i >= 2 ? 8 : 0);
-                    const float t = (full_tile || tok < ntok) ? s[mt][i] * p.scale_log2 : -INFINITY;
+                    const float t = (full_tile || tok < ((i & 1) ? lim1 : lim0)) ? s[mt][i] * p.scale_log2 : -INFINITY;
                     s[mt][i] = t;
                     if (i & 1) mx1 = fmaxf(mx1, t); else mx0 = fmaxf(mx0, t);
                 }
@@ -1026,9 +1049,14 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, x));
                 mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, x));
             }
-            const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
-            const float al0 = fast_exp2(m0 - mn0), al1 = fast_exp2(m1 - mn1);
+            const float mo0 = m0, mo1 = m1;
+            float mn0 = fmaxf(mo0, mx0), mn1 = fmaxf(mo1, mx1);
             m0 = mn0; m1 = mn1;
+            // a column that has seen no token yet (possible only for a later tile of a multi-token
+            // step) keeps m = -inf; exponentials are then taken against 0 so that they come out 0
+            mn0 = (mn0 == -INFINITY) ? 0.f : mn0;
+            mn1 = (mn1 == -INFINITY) ? 0.f : mn1;
+            const float al0 = fast_exp2(mo0 - mn0), al1 = fast_exp2(mo1 - mn1);
             l0 *= al0; l1 *= al1;
 #pragma unroll
             for (int dt = 0; dt < Lay::kDTiles; ++dt) {
@@ -1081,18 +1109,18 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             staging[(g0 + 1) * Lay::kStagePitch + d + 8] = o[dt][3];
         }
         __syncwarp();
-        uint16_t *out_rows = p.out + ((size_t)piece_r * p.num_q_heads + piece_h * G) * D;
+        uint16_t *out_rows = p.out + (size_t)piece_r * p.q_len * qi_stride + (size_t)piece_h * G * D;
         if (complete) {
 #pragma unroll
             for (int g = 0; g < kMaxGroup; ++g) {
                 const float lg = __shfl_sync(0xffffffffu, (g & 1) ? l1 : l0, g >> 1);
-                if (g < G && lane * 4 < D) {
+                if (g < ncols && lane * 4 < D) {
                     const float4 a = *(const float4 *)(staging + g * Lay::kStagePitch + lane * 4);
                     const float inv = 1.f / lg;
                     uint2 packed;
                     packed.x = pack_bf16x2(a.x * inv, a.y * inv);
                     packed.y = pack_bf16x2(a.z * inv, a.w * inv);
-                    *(uint2 *)(out_rows + (size_t)g * D + lane * 4) = packed;
+                    *(uint2 *)(out_rows + (size_t)(g / G) * qi_stride + (size_t)(g % G) * D + lane * 4) = packed;
                 }
             }
         } else {
@@ -1156,7 +1184,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 const int a = last0 ? 0 : 1, b = 1;
                 combine_small_pairs<D>(p.part_acc, p.part_ml, (last0 ? 1 : 0) + (last1 ? 1 : 0),
                                        pend_first[a], pend_last[a], pend_slot[a], pend_out[a],
-                                       pend_first[b], pend_last[b], pend_slot[b], pend_out[b], G, lane);
+                                       pend_first[b], pend_last[b], pend_slot[b], pend_out[b], ncols, G, qi_stride, lane);
             } else {
                 // stage 0's barrier has completed one phase per tile it carried; the ring is idle now
                 int bar_uses = (done + NS - 1) / NS;
@@ -1167,11 +1195,11 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     const int pieces = pend_last[k] - pend_first[k] + 1;
                     if (alive && pieces > kBulkMergeFrom)
                         alive = combine_partials_bulk<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k],
-                                                         pend_slot[k], G, lane, ring, NS * Lay::kStageBytes, bars,
+                                                         pend_slot[k], ncols, G, qi_stride, lane, ring, NS * Lay::kStageBytes, bars,
                                                          bar_uses, p.status);
                     else
                         combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k],
-                                            pend_slot[k], G, lane);
+                                            pend_slot[k], ncols, G, qi_stride, lane);
                 }
             }
         }

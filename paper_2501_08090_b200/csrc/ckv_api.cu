@@ -133,12 +133,12 @@ struct ckv_pool {
 
 namespace {
 
-template <int D, int W, int S>
+template <int D, int W, int S, bool kMulti>
 int32_t launch_attention(ckv_pool *pool, const ckv::AttnParams &ap, cudaStream_t stream)
 {
     using Lay = ckv::AttnLayout<D, W, S>;
     static thread_local int configured_device = -1;
-    auto kernel = ckv::paged_decode_attn_kernel<D, W, S>;
+    auto kernel = ckv::paged_decode_attn_kernel<D, W, S, kMulti>;
     if (configured_device != pool->device) {
         CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
         configured_device = pool->device;
@@ -213,7 +213,7 @@ template <int D, int W, int NS>
 int32_t launch_attention_noalloc(const CUtensorMap &tmap, const ckv::AttnParams &ap, cudaStream_t stream)
 {
     using Lay = ckv::AttnLayout<D, W, NS>;
-    auto kernel = ckv::paged_decode_attn_kernel<D, W, NS>;
+    auto kernel = ckv::paged_decode_attn_kernel<D, W, NS, false>;
     CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
     kernel<<<(ap.num_spans + W - 1) / W, Lay::kThreads, Lay::kSmemBytes, stream>>>(tmap, ap);
     CKV_CUDA(cudaGetLastError());
@@ -447,8 +447,12 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
         CKV_CUDA(cudaEventRecord(ev0, s));
     }
     int32_t rc;
-    if (c.head_dim == 128) rc = launch_attention<128, kWarps128, kStages128>(pool, ap, s);
-    else rc = launch_attention<64, kWarps64, kStages64>(pool, ap, s);
+    if (c.head_dim == 128)
+        rc = q_len > 1 ? launch_attention<128, kWarps128, kStages128, true>(pool, ap, s)
+                       : launch_attention<128, kWarps128, kStages128, false>(pool, ap, s);
+    else
+        rc = q_len > 1 ? launch_attention<64, kWarps64, kStages64, true>(pool, ap, s)
+                       : launch_attention<64, kWarps64, kStages64, false>(pool, ap, s);
     if (rc) return rc;
     if (ev1) CKV_CUDA(cudaEventRecord(ev1, s));
     pool->launches += 1;

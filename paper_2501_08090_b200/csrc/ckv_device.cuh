@@ -735,7 +735,9 @@ struct SpanCursor {
     }
 };
 
-template <int D, int W, int NS>
+// kMulti = false: one new token per request (every live column sees the whole context);
+// kMulti = true:  q_len > 1 new tokens, each column with its own causal limit.
+template <int D, int W, int NS, bool kMulti>
 __global__ void __launch_bounds__(W * 32, 1)
 paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnParams p)
 {
@@ -902,6 +904,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     SpanCursor cc;
     cc.r = st.r; cc.h = st.h; cc.tile = st.tile; cc.L = st.L; cc.tiles = st.tiles_r; cc.v = st.v;
     const int g0 = (lane & 3) * 2;               // first of the two group columns this lane accumulates
+    const int qi0 = g0 / G, qi1 = (g0 + 1) / G;  // the new tokens those two columns belong to
     uint32_t k_off[4], v_off[4];                 // ldmatrix lane offsets inside one page block
     {
         const int krow = (lane & 7) + ((lane >> 3) & 1) * 8;          // key row for matrices 0..3
@@ -965,10 +968,10 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             const int ntok = min(kTileTokens, piece_L - ti * kTileTokens);      // tokens of the context in this tile
             // Causality among the step's new tokens: column c (new token c / G) sees the context up to
             // and including its own position, i.e. vis_all + c / G tokens; every column sees vis_all.
-            const int vis_all = piece_L - p.q_len + 1;
+            const int vis_all = kMulti ? piece_L - p.q_len + 1 : piece_L;
             const bool full_tile = (ti + 1) * kTileTokens <= vis_all;
-            const int lim0 = min(ntok, vis_all + g0 / G - ti * kTileTokens);         // visible tokens of this tile,
-            const int lim1 = min(ntok, vis_all + (g0 + 1) / G - ti * kTileTokens);   // for this lane's two columns
+            const int lim0 = kMulti ? min(ntok, vis_all + qi0 - ti * kTileTokens) : ntok;   // visible tokens of this tile,
+            const int lim1 = kMulti ? min(ntok, vis_all + qi1 - ti * kTileTokens) : ntok;   // for this lane's two columns
             const int np = (ntok + kPageSize - 1) / kPageSize;
             const uint32_t sb = ring + slot * Lay::kStageBytes;
 
@@ -1054,8 +1057,10 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             m0 = mn0; m1 = mn1;
             // a column that has seen no token yet (possible only for a later tile of a multi-token
             // step) keeps m = -inf; exponentials are then taken against 0 so that they come out 0
-            mn0 = (mn0 == -INFINITY) ? 0.f : mn0;
-            mn1 = (mn1 == -INFINITY) ? 0.f : mn1;
+            if (kMulti) {
+                mn0 = (mn0 == -INFINITY) ? 0.f : mn0;
+                mn1 = (mn1 == -INFINITY) ? 0.f : mn1;
+            }
             const float al0 = fast_exp2(mo0 - mn0), al1 = fast_exp2(mo1 - mn1);
             l0 *= al0; l1 *= al1;
 #pragma unroll

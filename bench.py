@@ -387,6 +387,7 @@ def run_ours(args) -> None:
         if not args.no_sweep:
             line["latency_sweep"] = run_sweep(dev)
             line["local_autoscaler"] = run_autoscaler(line["latency_sweep"])
+            line["global_autoscaler"] = run_global_autoscaler(line["local_autoscaler"])
             line["kv_swap"] = run_swap(dev)
             line["multi_token_step"] = run_multi_token(dw)
         if not args.no_cpu_baseline:
@@ -492,6 +493,27 @@ def run_autoscaler(sweep: dict) -> dict:
         out["runs"].append({"itl_slo_ms": slo_ms, "peak_batch": int(tail.max()), "trough_batch": int(tail.min()),
                             "max_itl_ms": round(float(itl[200:].max()) / 1e3, 2),
                             "updates_to_first_halving": int(np.argmax(bp >= 1.0)) if (bp >= 1.0).any() else None})
+    return out
+
+
+def run_global_autoscaler(local: dict) -> dict:
+    """Section 5 on top of the measured instance: one batch instance serves (peak batch of the 2 s ITL run)
+    tokens every ITL; a queue of batch requests with a one-hour TTFT SLO (Section 6 "Workloads") is sized
+    by Algorithm 2 for a range of queue lengths, and an interactive pool is held at Theta = 1/3."""
+    from paper_2501_08090_b200 import binding
+    run = local["runs"][-1]
+    theta_tok_s = 0.75 * run["peak_batch"] / (run["max_itl_ms"] * 1e-3)       # saw-tooth mean: 3/4 of the peak
+    mu_o, sigma_o = 256.0, 192.0                                             # output tokens per request (synthetic)
+    out = {"tokens_per_s_per_instance": round(theta_tok_s), "mu_o": mu_o, "sigma_o": sigma_o, "z": 2.33,
+           "ttft_slo_s": 3600.0, "batch_queue": [], "interactive": []}
+    for queued in (10_000, 100_000, 1_000_000, 10_000_000):
+        n = binding.batch_autoscale([queued], [3600.0], mu_o, sigma_o, theta_tok_s, 0, 0, 1 << 16, z=2.33)
+        out["batch_queue"].append({"queued": queued, "instances": n,
+                                   "wait_s": round(binding.waiting_time(queued - 1, mu_o, sigma_o, theta_tok_s * n, 2.33), 1)})
+    total = 9
+    for busy in (3, 5, 8, 4, 1):
+        total = binding.interactive_autoscale(busy, total, 1.0 / 3.0, 0.05)
+        out["interactive"].append({"busy": busy, "instances": total})
     return out
 
 

@@ -65,6 +65,58 @@ int32_t local_autoscaler_simulate(const ckv_autoscaler_config *cfg, double initi
                                   double *out_max_bs, int32_t *out_batch, double *out_itl_us,
                                   double *out_backpressure);
 
+/* ------------------------------------------------------------------------------------------
+ * Global autoscaler primitives (Section 5 "Global Autoscaler").  Host-only.
+ * ------------------------------------------------------------------------------------------ */
+
+/*
+ * Request groups (Section 5.3, "Request Group Creation"): cluster the queued requests by TTFT SLO
+ * with 1-D k-means.  Centroids start at evenly spaced quantiles of the sorted values and Lloyd
+ * iterations run to a fixed point (at most 100); groups are numbered by increasing centroid, ties
+ * in distance go to the lower centroid.  k is clamped to [1, n].
+ *   out_group [n]: group of every request;  out_centroids [k] (may be NULL).
+ */
+int32_t global_request_groups(const double *ttft_slos, int32_t n, int32_t k, int32_t *out_group,
+                              double *out_centroids);
+
+/*
+ * Waiting time of a request with `requests_ahead` requests before it in the queue (Eq. 1): the
+ * output tokens ahead are a sum of i.i.d. lengths with fitted mean mu_o and deviation sigma_o
+ * (normal by the CLT), served at a constant token throughput:
+ *   W = (requests_ahead * mu_o + z * sigma_o * sqrt(requests_ahead)) / throughput
+ * z = 0 gives the mean estimate; z > 0 a conservative quantile.
+ */
+int32_t global_waiting_time(int32_t requests_ahead, double mu_o, double sigma_o, double throughput, double z,
+                            double *out_seconds);
+
+/*
+ * Batch backpressure (Section 5.3): BBP = number of request groups whose estimated waiting time
+ * exceeds their TTFT deadline.  Groups are given in service order (increasing TTFT SLO, FCFS
+ * inside); group g's waiting time is that of its LAST request: requests_ahead = requests of the
+ * earlier groups + counts[g] - 1, at throughput_per_instance * instances.  deadlines[g] is the
+ * time the group still has (its TTFT SLO minus the age of its oldest request).
+ */
+int32_t global_batch_backpressure(const int32_t *counts, const double *deadlines, int32_t n_groups, double mu_o,
+                                  double sigma_o, double throughput_per_instance, int32_t instances, double z,
+                                  int32_t *out_bbp);
+
+/*
+ * Algorithm 2 (Batch Instance Autoscaling): starting from the instances already dispatched (at
+ * least one), add one instance at a time until BBP = 0 or max_instances is reached; with an empty
+ * queue, retire every batch instance once no request is active on them.
+ */
+int32_t global_batch_autoscale(const int32_t *counts, const double *deadlines, int32_t n_groups, double mu_o,
+                               double sigma_o, double throughput_per_instance, int32_t current_instances,
+                               int32_t active_requests, int32_t max_instances, double z, int32_t *out_instances);
+
+/*
+ * Interactive autoscaling (Section 5.2): IBP = instances running interactive requests / (mixed +
+ * interactive instances).  While IBP stays inside [theta - delta, theta + delta] the count is
+ * kept; outside the band it becomes ceil(busy / theta), never below `busy` or `floor_instances`.
+ */
+int32_t global_interactive_autoscale(int32_t busy, int32_t total, double theta, double delta,
+                                     int32_t floor_instances, int32_t *out_total);
+
 #ifdef __cplusplus
 }
 #endif

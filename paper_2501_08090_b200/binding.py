@@ -29,6 +29,8 @@ EXPORTS = (
     "kv_append_multi", "decode_attention_multi",
     "local_autoscaler_instance_slo", "local_autoscaler_create", "local_autoscaler_destroy",
     "local_autoscaler_update", "local_autoscaler_get", "local_autoscaler_simulate",
+    "global_request_groups", "global_waiting_time", "global_batch_backpressure", "global_batch_autoscale",
+    "global_interactive_autoscale",
 )
 
 
@@ -92,6 +94,14 @@ def _load() -> ctypes.CDLL:
     lib.local_autoscaler_get.restype = i32; lib.local_autoscaler_get.argtypes = [vp, f64p]
     lib.local_autoscaler_simulate.restype = i32
     lib.local_autoscaler_simulate.argtypes = [acfgp, f64, i32, vp, vp, f64, i32, i32, vp, vp, vp, vp]
+    lib.global_request_groups.restype = i32; lib.global_request_groups.argtypes = [vp, i32, i32, vp, vp]
+    lib.global_waiting_time.restype = i32; lib.global_waiting_time.argtypes = [i32, f64, f64, f64, f64, f64p]
+    lib.global_batch_backpressure.restype = i32
+    lib.global_batch_backpressure.argtypes = [vp, vp, i32, f64, f64, f64, i32, f64, i32p]
+    lib.global_batch_autoscale.restype = i32
+    lib.global_batch_autoscale.argtypes = [vp, vp, i32, f64, f64, f64, i32, i32, i32, f64, i32p]
+    lib.global_interactive_autoscale.restype = i32
+    lib.global_interactive_autoscale.argtypes = [i32, i32, f64, f64, i32, i32p]
     lib.ckv_launch_count.restype = i64; lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_last_error.restype = ctypes.c_char_p; lib.ckv_last_error.argtypes = []
     return lib
@@ -381,3 +391,53 @@ def autoscaler_simulate(itl_slo_us: float, initial_max_bs: float, batch_sizes, u
     if rc != CKV_OK:
         raise CkvError(rc, "local_autoscaler_simulate: bad argument")
     return o_bs, o_b, o_itl, o_bp
+
+
+# ----------------------------------------------------------------------------- global autoscaler
+
+def _rc(rc: int, what: str) -> None:
+    if rc != CKV_OK:
+        raise CkvError(rc, what + ": bad argument")
+
+
+def request_groups(ttft_slos, k: int):
+    """(group index of every request, centroids in increasing order): 1-D k-means on TTFT SLOs."""
+    x = np.ascontiguousarray(ttft_slos, dtype=np.float64)
+    kk = max(1, min(int(k), int(x.size)))
+    grp = np.zeros(x.size, dtype=np.int32)
+    cent = np.zeros(kk, dtype=np.float64)
+    _rc(lib.global_request_groups(x.ctypes.data, int(x.size), int(k), grp.ctypes.data, cent.ctypes.data), "global_request_groups")
+    return grp, cent
+
+
+def waiting_time(requests_ahead: int, mu_o: float, sigma_o: float, throughput: float, z: float = 0.0) -> float:
+    out = ctypes.c_double(0.0)
+    _rc(lib.global_waiting_time(int(requests_ahead), float(mu_o), float(sigma_o), float(throughput), float(z),
+                                ctypes.byref(out)), "global_waiting_time")
+    return out.value
+
+
+def batch_backpressure(counts, deadlines, mu_o, sigma_o, throughput_per_instance, instances, z=0.0) -> int:
+    c = np.ascontiguousarray(counts, dtype=np.int32); d = np.ascontiguousarray(deadlines, dtype=np.float64)
+    out = ctypes.c_int32(0)
+    _rc(lib.global_batch_backpressure(c.ctypes.data, d.ctypes.data, int(c.size), float(mu_o), float(sigma_o),
+                                      float(throughput_per_instance), int(instances), float(z), ctypes.byref(out)),
+        "global_batch_backpressure")
+    return out.value
+
+
+def batch_autoscale(counts, deadlines, mu_o, sigma_o, throughput_per_instance, current_instances,
+                    active_requests, max_instances, z=0.0) -> int:
+    c = np.ascontiguousarray(counts, dtype=np.int32); d = np.ascontiguousarray(deadlines, dtype=np.float64)
+    out = ctypes.c_int32(0)
+    _rc(lib.global_batch_autoscale(c.ctypes.data, d.ctypes.data, int(c.size), float(mu_o), float(sigma_o),
+                                   float(throughput_per_instance), int(current_instances), int(active_requests),
+                                   int(max_instances), float(z), ctypes.byref(out)), "global_batch_autoscale")
+    return out.value
+
+
+def interactive_autoscale(busy: int, total: int, theta: float, delta: float, floor: int = 1) -> int:
+    out = ctypes.c_int32(0)
+    _rc(lib.global_interactive_autoscale(int(busy), int(total), float(theta), float(delta), int(floor),
+                                         ctypes.byref(out)), "global_interactive_autoscale")
+    return out.value

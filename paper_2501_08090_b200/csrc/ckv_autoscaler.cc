@@ -134,3 +134,119 @@ int32_t local_autoscaler_simulate(const ckv_autoscaler_config *cfg, double initi
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------
+// Global autoscaler primitives (Section 5).
+// ------------------------------------------------------------------------------------------
+#include <vector>
+
+namespace {
+double wait_seconds(int32_t ahead, double mu, double sigma, double thr, double z)
+{
+    if (ahead <= 0) return 0.0;
+    return ((double)ahead * mu + z * sigma * std::sqrt((double)ahead)) / thr;
+}
+
+int32_t bbp_of(const int32_t *counts, const double *deadlines, int32_t n, double mu, double sigma, double thr, double z)
+{
+    int32_t bbp = 0;
+    long long ahead = 0;
+    for (int32_t g = 0; g < n; ++g) {
+        if (counts[g] <= 0) continue;
+        if (wait_seconds((int32_t)(ahead + counts[g] - 1), mu, sigma, thr, z) > deadlines[g]) ++bbp;
+        ahead += counts[g];
+    }
+    return bbp;
+}
+}  // namespace
+
+extern "C" {
+
+int32_t global_request_groups(const double *ttft_slos, int32_t n, int32_t k, int32_t *out_group, double *out_centroids)
+{
+    if (!ttft_slos || n < 1 || k < 1 || !out_group) return kInval;
+    k = std::min(k, n);
+    std::vector<double> sorted(ttft_slos, ttft_slos + n);
+    std::sort(sorted.begin(), sorted.end());
+    std::vector<double> cent(k), next(k);
+    for (int32_t j = 0; j < k; ++j) cent[j] = sorted[std::min<long long>(n - 1, (long long)(2 * j + 1) * n / (2 * k))];
+    std::vector<int32_t> assign(n, 0), cur(n);
+    for (int it = 0; it < 100; ++it) {
+        for (int32_t i = 0; i < n; ++i) {
+            int32_t best = 0;
+            double bd = std::fabs(ttft_slos[i] - cent[0]);
+            for (int32_t j = 1; j < k; ++j) {
+                const double d = std::fabs(ttft_slos[i] - cent[j]);
+                if (d < bd) { bd = d; best = j; }
+            }
+            cur[i] = best;
+        }
+        for (int32_t j = 0; j < k; ++j) {
+            double sum = 0.0;
+            long long cnt = 0;
+            for (int32_t i = 0; i < n; ++i) if (cur[i] == j) { sum += ttft_slos[i]; ++cnt; }
+            next[j] = cnt ? sum / (double)cnt : cent[j];
+        }
+        const bool fixed = (cur == assign) && (next == cent);
+        assign = cur;
+        cent = next;
+        if (fixed) break;
+    }
+    std::vector<int32_t> rank(k);
+    for (int32_t j = 0; j < k; ++j) rank[j] = j;
+    std::stable_sort(rank.begin(), rank.end(), [&](int32_t a, int32_t b) { return cent[a] < cent[b]; });
+    std::vector<int32_t> relabel(k);
+    for (int32_t r = 0; r < k; ++r) relabel[rank[r]] = r;
+    for (int32_t i = 0; i < n; ++i) out_group[i] = relabel[assign[i]];
+    if (out_centroids) for (int32_t r = 0; r < k; ++r) out_centroids[r] = cent[rank[r]];
+    return kOk;
+}
+
+int32_t global_waiting_time(int32_t requests_ahead, double mu_o, double sigma_o, double throughput, double z,
+                            double *out_seconds)
+{
+    if (!out_seconds || !(throughput > 0.0) || mu_o < 0.0 || sigma_o < 0.0 || requests_ahead < 0) return kInval;
+    *out_seconds = wait_seconds(requests_ahead, mu_o, sigma_o, throughput, z);
+    return kOk;
+}
+
+int32_t global_batch_backpressure(const int32_t *counts, const double *deadlines, int32_t n_groups, double mu_o,
+                                  double sigma_o, double throughput_per_instance, int32_t instances, double z,
+                                  int32_t *out_bbp)
+{
+    if (!counts || !deadlines || n_groups < 0 || !out_bbp || instances < 1 || !(throughput_per_instance > 0.0)) return kInval;
+    *out_bbp = bbp_of(counts, deadlines, n_groups, mu_o, sigma_o, throughput_per_instance * instances, z);
+    return kOk;
+}
+
+int32_t global_batch_autoscale(const int32_t *counts, const double *deadlines, int32_t n_groups, double mu_o,
+                               double sigma_o, double throughput_per_instance, int32_t current_instances,
+                               int32_t active_requests, int32_t max_instances, double z, int32_t *out_instances)
+{
+    if (!out_instances || n_groups < 0 || (n_groups > 0 && (!counts || !deadlines))) return kInval;
+    if (current_instances < 0 || active_requests < 0 || max_instances < 1 || !(throughput_per_instance > 0.0)) return kInval;
+    long long queued = 0;
+    for (int32_t g = 0; g < n_groups; ++g) queued += std::max(0, counts[g]);
+    if (queued == 0) {
+        *out_instances = active_requests == 0 ? 0 : current_instances;
+        return kOk;
+    }
+    int32_t n = std::max(1, current_instances);
+    while (n < max_instances && bbp_of(counts, deadlines, n_groups, mu_o, sigma_o, throughput_per_instance * n, z) > 0) ++n;
+    *out_instances = n;
+    return kOk;
+}
+
+int32_t global_interactive_autoscale(int32_t busy, int32_t total, double theta, double delta, int32_t floor_instances,
+                                     int32_t *out_total)
+{
+    if (!out_total || busy < 0 || total < 0 || !(theta > 0.0) || theta > 1.0 || delta < 0.0 || floor_instances < 0) return kInval;
+    total = std::max(std::max(total, floor_instances), 1);
+    const double ibp = (double)busy / (double)total;
+    if (ibp >= theta - delta && ibp <= theta + delta) { *out_total = total; return kOk; }
+    const int32_t want = (int32_t)std::ceil((double)busy / theta - 1e-12);
+    *out_total = std::max(std::max(floor_instances, busy), want);
+    return kOk;
+}
+
+}  // extern "C"

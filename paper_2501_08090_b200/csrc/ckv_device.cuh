@@ -21,6 +21,7 @@ constexpr int kMaxGroup = 8;         // query heads per KV head handled by one M
 constexpr int kMaxSpans = 2048;      // upper bound on the partition width (one span per warp)
 constexpr int kMaxBatch = 8192;
 constexpr int kBulkMergeFrom = 4;    // merges of more partials than this go through shared memory
+constexpr int kTreeFrom = 12;        // pairs cut into more partials than this are merged in two levels
 
 constexpr uint32_t kStatusBadLength = 1u;
 constexpr uint32_t kStatusBadPage = 2u;
@@ -37,6 +38,14 @@ constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // bound of every d
 #define CKV_PIECE_COST_TILES 2
 #endif
 constexpr int kPieceCostTiles = CKV_PIECE_COST_TILES;
+
+// Partials per first-level group of a two-level merge of n partials: a power of two near sqrt(n).
+__host__ __device__ __forceinline__ int merge_group_size(int n)
+{
+    int sub = 8;
+    while (sub * sub < n) sub *= 2;
+    return sub;
+}
 
 struct PlanHeader {
     int32_t total_units;
@@ -320,6 +329,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
 // Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
 // start while its predecessor in the stream still runs.  grid_dependency_wait() blocks until the
 // predecessor has completed and its writes are visible; without the attribute it returns at once.
+// Start fetching a tensor map (a kernel parameter) so that the first tile load does not wait for it.
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
 __device__ __forceinline__ void grid_dependency_wait()
 {
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -463,13 +478,48 @@ struct AttnParams {
 // Merge the partials of one (request, kv head) that spans s_first..s_last hold, and write its bf16
 // output rows.  Run by one whole warp (the last one to arrive for that pair).  Loads are issued in
 // batches so the merge costs a few L2 round trips, not one per partial.
+//
+// Which partials: numbers i0, i0 + stride, ... (`pieces` of them) of the pair, where partial i lives
+// in slot_first (i = 0) or in the first slot of span s_first + i.  Where the result goes: to
+// dst_acc / dst_ml as one merged partial (same format, not normalised) if dst_acc is not NULL,
+// else normalised to the bf16 output rows.
+struct MergeSel {
+    int s_first, slot_first;   // the pair's first span and the slot of its partial 0
+    int i0, stride, pieces;    // the partials to merge
+    __device__ __forceinline__ int slot_of(int t) const
+    {
+        const int i = i0 + t * stride;
+        return i == 0 ? slot_first : 2 * (s_first + i);
+    }
+};
+
+template <int D>
+__device__ __forceinline__ void store_merged(const float4 (&acc)[kMaxGroup], const float (&mstar)[kMaxGroup],
+                                             const float (&lsum)[kMaxGroup], float *dst_acc, float *dst_ml,
+                                             uint16_t *out_rows, int ncols, int G, int qi_stride, int lane)
+{
+#pragma unroll
+    for (int g = 0; g < kMaxGroup; ++g) {
+        if (dst_acc != nullptr) {
+            if (g < ncols && lane * 4 < D) *(float4 *)(dst_acc + g * D + lane * 4) = acc[g];
+            if (lane == 0) { dst_ml[g] = mstar[g]; dst_ml[kMaxGroup + g] = lsum[g]; }
+        } else if (g < ncols && lane * 4 < D) {
+            const float inv = 1.f / lsum[g];
+            uint2 packed;
+            packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
+            packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
+            *(uint2 *)(out_rows + (size_t)(g / G) * qi_stride + (size_t)(g % G) * D + lane * 4) = packed;
+        }
+    }
+}
+
 template <int D>
 __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
-                                              uint16_t *out_rows, int s_first, int s_last, int slot_first, int ncols, int G,
-                                              int qi_stride, int lane)
+                                              uint16_t *out_rows, const MergeSel sel, float *dst_acc, float *dst_ml,
+                                              int ncols, int G, int qi_stride, int lane)
 {
-    const int pieces = s_last - s_first + 1;
-    auto slot_of = [&](int i) { return i == 0 ? slot_first : 2 * (s_first + i); };
+    const int pieces = sel.pieces;
+    auto slot_of = [&](int t) { return sel.slot_of(t); };
 
     // (m, l) of the partial this lane owns in the first round of 32; usually the only round
     float mi[kMaxGroup], li[kMaxGroup];
@@ -508,7 +558,9 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
             if (base > 0) load_ml(base + lane);
 #pragma unroll
             for (int g = 0; g < kMaxGroup; ++g) {
-                f_mine[g] = fast_exp2(mi[g] - mstar[g]);
+                // a column may have seen no token in any of these partials (a group of a multi-token
+                // step's two-level merge): its maximum stays -inf and its factors are 0
+                f_mine[g] = fast_exp2(mi[g] - (mstar[g] == -INFINITY ? 0.f : mstar[g]));
                 lsum[g] += f_mine[g] * li[g];
             }
         }
@@ -530,14 +582,8 @@ __device__ __noinline__ void combine_partials(const float *__restrict__ part_acc
     for (int g = 0; g < kMaxGroup; ++g) {
 #pragma unroll
         for (int x = 16; x > 0; x >>= 1) lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], x);
-        if (g < ncols && lane * 4 < D) {
-            const float inv = 1.f / lsum[g];
-            uint2 packed;
-            packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
-            packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
-            *(uint2 *)(out_rows + (size_t)(g / G) * qi_stride + (size_t)(g % G) * D + lane * 4) = packed;
-        }
     }
+    store_merged<D>(acc, mstar, lsum, dst_acc, dst_ml, out_rows, ncols, G, qi_stride, lane);
 }
 
 // Merge of up to two (request, kv head) pairs with at most four partials each -- the usual case at
@@ -619,12 +665,12 @@ __device__ __noinline__ void combine_small_pairs(const float *__restrict__ part_
 // bounded wait gave up.
 template <int D>
 __device__ __noinline__ bool combine_partials_bulk(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
-                                                   uint16_t *out_rows, int s_first, int s_last, int slot_first, int ncols,
-                                                   int G, int qi_stride, int lane, uint32_t ring, int ring_bytes, uint32_t bar, int &uses,
-                                                   uint32_t *status)
+                                                   uint16_t *out_rows, const MergeSel sel, float *dst_acc, float *dst_ml,
+                                                   int ncols, int G, int qi_stride, int lane, uint32_t ring, int ring_bytes,
+                                                   uint32_t bar, int &uses, uint32_t *status)
 {
-    const int pieces = s_last - s_first + 1;
-    auto slot_of = [&](int i) { return i == 0 ? slot_first : 2 * (s_first + i); };
+    const int pieces = sel.pieces;
+    auto slot_of = [&](int t) { return sel.slot_of(t); };
     const int piece_bytes = ncols * D * 4;                   // the live rows of a partial are contiguous
     const int cap = min(32, ring_bytes / piece_bytes);
 
@@ -657,11 +703,14 @@ __device__ __noinline__ bool combine_partials_bulk(const float *__restrict__ par
             float mx = mi[g];
 #pragma unroll
             for (int x = 16; x > 0; x >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, x));
-            const float mnew = fmaxf(mstar[g], mx);           // finite: every partial holds at least one token
-            const float rescale = fast_exp2(mstar[g] - mnew);
+            const float mnew = fmaxf(mstar[g], mx);
+            // -inf only while no partial so far has seen a token for this column (a multi-token step):
+            // exponentials are then taken against 0 and come out 0
+            const float mref = mnew == -INFINITY ? 0.f : mnew;
+            const float rescale = fast_exp2(mstar[g] - mref);
             mstar[g] = mnew;
             acc[g].x *= rescale; acc[g].y *= rescale; acc[g].z *= rescale; acc[g].w *= rescale;
-            f_mine[g] = fast_exp2(mi[g] - mnew);              // lanes without a partial: exp2(-inf) = 0
+            f_mine[g] = fast_exp2(mi[g] - mref);              // lanes without a partial: exp2(-inf) = 0
             lsum[g] = lsum[g] * rescale + f_mine[g] * li[g];
         }
         ok = mbar_wait_bounded(bar, uses & 1, status);
@@ -685,14 +734,8 @@ __device__ __noinline__ bool combine_partials_bulk(const float *__restrict__ par
     for (int g = 0; g < kMaxGroup; ++g) {
 #pragma unroll
         for (int x = 16; x > 0; x >>= 1) lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], x);
-        if (g < ncols && lane * 4 < D) {
-            const float inv = 1.f / lsum[g];
-            uint2 packed;
-            packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
-            packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
-            *(uint2 *)(out_rows + (size_t)(g / G) * qi_stride + (size_t)(g % G) * D + lane * 4) = packed;
-        }
     }
+    store_merged<D>(acc, mstar, lsum, dst_acc, dst_ml, out_rows, ncols, G, qi_stride, lane);
     return true;
 }
 
@@ -756,6 +799,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     unsigned long long t_start = 0;
     if (lane == 0) {
         t_start = global_timer_ns();
+        prefetch_tensormap(&tmap);
         for (int s = 0; s < NS; ++s) mbar_init(bars + s * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
@@ -1163,48 +1207,92 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 
     if (lane == 0) p.trace[span * 8 + 2] = global_timer_ns();
 
-    // ---- arrivals: whichever warp arrives last for a (request, kv head) merges its partials (wait-free)
+    // ---- arrivals: whichever warp arrives last for a (request, kv head) merges its partials (wait-free).
+    // A pair cut into more than kTreeFrom partials is merged in two levels: its partials form groups
+    // of `sub` consecutive ones, each with a counter of its own (kept in arrivals[] at the pair's
+    // interior spans, which no other pair uses); the last arriver of a group folds it into the slot
+    // of the group's first partial and then arrives for the pair, and the last group to arrive folds
+    // the group results.  Groups complete while other warps are still streaming, so the tail of the
+    // launch holds one short merge instead of one long one.
     if (pend_first[0] >= 0 || pend_first[1] >= 0) {
+        int n_part[2], sub[2], grp[2], grp_cnt[2], n_grp[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            n_part[k] = pend_first[k] >= 0 ? pend_last[k] - pend_first[k] + 1 : 0;
+            sub[k] = 0; grp[k] = 0; grp_cnt[k] = n_part[k]; n_grp[k] = 1;
+            if (n_part[k] > kTreeFrom) {
+                sub[k] = merge_group_size(n_part[k]);
+                grp[k] = (span - pend_first[k]) / sub[k];
+                n_grp[k] = (n_part[k] + sub[k] - 1) / sub[k];
+                grp_cnt[k] = min(sub[k], n_part[k] - grp[k] * sub[k]);
+            }
+        }
         __threadfence();
         __syncwarp();
         int prior0 = 0, prior1 = 0;
         if (lane == 0) {                          // both round trips in flight together
-            if (pend_first[0] >= 0) prior0 = atomicAdd(p.arrivals + pend_first[0], 1);
-            if (pend_first[1] >= 0) prior1 = atomicAdd(p.arrivals + pend_first[1], 1);
+            if (pend_first[0] >= 0) prior0 = atomicAdd(p.arrivals + pend_first[0] + (sub[0] ? 1 + grp[0] : 0), 1);
+            if (pend_first[1] >= 0) prior1 = atomicAdd(p.arrivals + pend_first[1] + (sub[1] ? 1 + grp[1] : 0), 1);
         }
         prior0 = __shfl_sync(0xffffffffu, prior0, 0);
         prior1 = __shfl_sync(0xffffffffu, prior1, 0);
-        const bool last0 = pend_first[0] >= 0 && prior0 == pend_last[0] - pend_first[0];
-        const bool last1 = pend_first[1] >= 0 && prior1 == pend_last[1] - pend_first[1];
-        if (last0 || last1) {
+        bool last[2];
+        last[0] = pend_first[0] >= 0 && prior0 == grp_cnt[0] - 1;
+        last[1] = pend_first[1] >= 0 && prior1 == grp_cnt[1] - 1;
+        if (last[0] || last[1]) {
             __threadfence();
             if (lane == 0) {                      // counters are ready for the next launch
-                if (last0) p.arrivals[pend_first[0]] = 0;
-                if (last1) p.arrivals[pend_first[1]] = 0;
+                if (last[0]) p.arrivals[pend_first[0] + (sub[0] ? 1 + grp[0] : 0)] = 0;
+                if (last[1]) p.arrivals[pend_first[1] + (sub[1] ? 1 + grp[1] : 0)] = 0;
             }
-            const int pieces0 = last0 ? pend_last[0] - pend_first[0] + 1 : 0;
-            const int pieces1 = last1 ? pend_last[1] - pend_first[1] + 1 : 0;
-            if (pieces0 <= kBulkMergeFrom && pieces1 <= kBulkMergeFrom) {
+            // stage 0's barrier has completed one phase per tile it carried; the ring is idle now
+            int bar_uses = (done + NS - 1) / NS;
+            auto merge = [&](int k, const MergeSel sel, float *dst_acc, float *dst_ml) {
+                if (alive && sel.pieces > kBulkMergeFrom) {
+                    fence_proxy_async();          // partials written through the generic proxy, read by bulk copies
+                    alive = combine_partials_bulk<D>(p.part_acc, p.part_ml, pend_out[k], sel, dst_acc, dst_ml, ncols, G,
+                                                     qi_stride, lane, ring, NS * Lay::kStageBytes, bars, bar_uses, p.status);
+                } else {
+                    combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], sel, dst_acc, dst_ml, ncols, G, qi_stride, lane);
+                }
+            };
+            // first level of the two-level merges
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                if (!last[k] || sub[k] == 0) continue;
+                MergeSel sel;
+                sel.s_first = pend_first[k]; sel.slot_first = pend_slot[k];
+                sel.i0 = grp[k] * sub[k]; sel.stride = 1; sel.pieces = grp_cnt[k];
+                const int dst_slot = sel.slot_of(0);
+                merge(k, sel, p.part_acc + (size_t)dst_slot * kMaxGroup * D, p.part_ml + dst_slot * 2 * kMaxGroup);
+                __threadfence();
+                __syncwarp();
+                int prior = 0;
+                if (lane == 0) prior = atomicAdd(p.arrivals + pend_first[k], 1);
+                prior = __shfl_sync(0xffffffffu, prior, 0);
+                last[k] = prior == n_grp[k] - 1;
+                if (last[k]) {
+                    __threadfence();
+                    if (lane == 0) p.arrivals[pend_first[k]] = 0;
+                }
+            }
+            // final merges
+            const int fin0 = last[0] ? (sub[0] ? n_grp[0] : n_part[0]) : 0;
+            const int fin1 = last[1] ? (sub[1] ? n_grp[1] : n_part[1]) : 0;
+            if ((last[0] || last[1]) && fin0 <= kBulkMergeFrom && fin1 <= kBulkMergeFrom && sub[0] == 0 && sub[1] == 0) {
                 // the usual case: one or two short merges, done together
-                const int a = last0 ? 0 : 1, b = 1;
-                combine_small_pairs<D>(p.part_acc, p.part_ml, (last0 ? 1 : 0) + (last1 ? 1 : 0),
+                const int a = last[0] ? 0 : 1, b = 1;
+                combine_small_pairs<D>(p.part_acc, p.part_ml, (last[0] ? 1 : 0) + (last[1] ? 1 : 0),
                                        pend_first[a], pend_last[a], pend_slot[a], pend_out[a],
                                        pend_first[b], pend_last[b], pend_slot[b], pend_out[b], ncols, G, qi_stride, lane);
             } else {
-                // stage 0's barrier has completed one phase per tile it carried; the ring is idle now
-                int bar_uses = (done + NS - 1) / NS;
-                fence_proxy_async();              // partials written through the generic proxy, read by bulk copies
 #pragma unroll
                 for (int k = 0; k < 2; ++k) {
-                    if (!(k == 0 ? last0 : last1)) continue;
-                    const int pieces = pend_last[k] - pend_first[k] + 1;
-                    if (alive && pieces > kBulkMergeFrom)
-                        alive = combine_partials_bulk<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k],
-                                                         pend_slot[k], ncols, G, qi_stride, lane, ring, NS * Lay::kStageBytes, bars,
-                                                         bar_uses, p.status);
-                    else
-                        combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], pend_first[k], pend_last[k],
-                                            pend_slot[k], ncols, G, qi_stride, lane);
+                    if (!last[k]) continue;
+                    MergeSel sel;
+                    sel.s_first = pend_first[k]; sel.slot_first = pend_slot[k];
+                    sel.i0 = 0; sel.stride = sub[k] ? sub[k] : 1; sel.pieces = k == 0 ? fin0 : fin1;
+                    merge(k, sel, nullptr, nullptr);
                 }
             }
         }

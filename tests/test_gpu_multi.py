@@ -56,6 +56,17 @@ def test_multi_token_step_matches_oracle(q_len, Hq, Hkv, d):
     run_case(q_len, Hq, Hkv, d, lens, seed=q_len * 100 + Hq, partitions=(None, 1, 11, 2048))
 
 
+@pytest.mark.parametrize("n_tiles", [12, 13, 16, 17, 24, 25, 64, 65, 80, 257, 300])
+@pytest.mark.parametrize("q_len", [1, 4])
+def test_two_level_merge_of_many_partials(n_tiles, q_len):
+    """One request cut into one partial per tile (2048 spans for a handful of units): group sizes 8, 16 and
+    32, full and ragged last groups, a last group of one, and (q_len 4) groups in which the early new
+    tokens see nothing at all."""
+    for tail in (1, 32):
+        run_case(q_len, 2, 1, 128, [(n_tiles - 1) * 32 + tail], seed=n_tiles + tail, partitions=(2048,))
+    run_case(q_len, 4, 2, 64, [(n_tiles - 1) * 32 + 7, 40, n_tiles * 32], seed=n_tiles, partitions=(2048, 700))
+
+
 def test_new_tokens_straddling_every_tile_boundary():
     for L in range(30, 40):                                    # the 4 new tokens walk across the 32-token boundary
         run_case(4, 4, 2, 128, [L, 4, L + 32], seed=L)

@@ -156,38 +156,18 @@ int32_t decode_attention_multi(ckv_pool *pool, int32_t layer, int32_t batch, int
 /*
  * The split-KV partition decode_attention uses for these lengths, copied to the host for
  * inspection (runs a small kernel and synchronises `stream`; decode_attention itself derives the
- * same partition inside its attention kernel and launches no plan kernel).  A "tile" is
- * ckv_tile_tokens() consecutive tokens of one (request, KV head).  Work is laid out on an axis of
- * units, request-major then KV head: each (request, KV head) contributes CKV_PIECE_COST_TILES (2)
- * overhead units followed by one unit per tile.  The axis is cut into cells.  Cell s < num_spans
- * -- the first work of warp s -- owns the tiles whose units fall in
- * [s*units_per_span, min((s+1)*units_per_span, S)), S = min(num_spans*units_per_span, total_units).
- * With a dynamic share set (ckv_set_dynamic) units_per_span is chosen so that this share of the
- * axis is left over behind S; it is cut into dyn_cells[0] cells of dyn_pitch[0] units followed by
- * dyn_cells[1] cells of dyn_pitch[1] units, which warps claim in order as they finish.
- *   h_header[16]  : total_units, units_per_span, num_spans, number of spans with a non-empty range,
- *                   num_cells, dyn_cells[2], dyn_pitch[2], 7 reserved
- *   h_span_start  : int32 [num_cells][4] = request, kv head, first tile within that
- *                   (request, kv head), unit index of that tile; -1s if the cell holds no tile
- * h_span_start must hold 4*ckv_max_cells() ints.  Errors: CKV_EINVAL, CKV_ECUDA.
+ * same partition inside its attention kernel and launches no plan kernel).  A "tile" is 32
+ * consecutive tokens of one (request, KV head).  Work is laid out on an axis of units,
+ * request-major then KV head: each (request, KV head) contributes CKV_PIECE_COST_TILES (2)
+ * overhead units followed by one unit per tile.  Span s -- the work of one warp -- owns the tiles
+ * whose units fall in [s*units_per_span, min((s+1)*units_per_span, total_units)).
+ *   h_header[4]   : total_units, units_per_span, num_spans, number of spans with a non-empty range
+ *   h_span_start  : int32 [num_spans][4] = request, kv head, first tile within that
+ *                   (request, kv head), unit index of that tile; -1s if the span holds no tile
+ * h_span_start must hold 4*ckv_get_partition() ints.  Errors: CKV_EINVAL, CKV_ECUDA.
  */
 int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *stream,
                     int32_t *h_header, int32_t *h_span_start);
-
-/* Upper bound on the number of cells of a partition; tokens per tile. */
-int32_t ckv_max_cells(void);
-int32_t ckv_tile_tokens(void);
-
-/* Dynamic share of the partition.  SMs do not all stream from HBM at the same rate (the spread
- * between the fastest and the slowest is about a quarter on a B200), so a partition into equal
- * spans ends when the slowest SM ends.  With permille > 0 that many thousandths of the work are
- * held back from the spans and cut into small cells -- two thirds of it into cells of
- * cell_units_1 units, the rest into cells of cell_units_2 <= cell_units_1 units (0: one size
- * only) -- which warps claim from a counter when they have finished what they hold, so faster SMs
- * take more.  Which warp computes a cell never changes the result: cells, their partial results
- * and the order in which these are merged are fixed by the lengths alone.  Problems with fewer
- * than 8 units per span stay static.  0 <= permille <= 900.  Errors: CKV_EINVAL. */
-int32_t ckv_set_dynamic(ckv_pool *pool, int32_t permille, int32_t cell_units_1, int32_t cell_units_2);
 
 /* Number of spans the partition is balanced over (default: warps per CTA x number of SMs).
  * Setting it changes only how the context is split, never the result beyond fp32 summation
@@ -201,8 +181,11 @@ int32_t ckv_get_partition(const ckv_pool *pool);
  * The attention prologue reads d_seq_lens and d_block_tables BEFORE that wait, so with overlap on
  * they must not be produced by the kernel that immediately precedes decode_attention in the
  * stream (tables copied by a memcpy, or written by any earlier kernel, are fine -- the usual case,
- * since a serving engine uploads them once per iteration).  Turning overlap off restores plain
- * stream order.  Errors: CKV_EINVAL. */
+ * since a serving engine uploads them once per iteration).  decode_step, being the only writer of
+ * its layer's pool, also starts its first KV tile loads before that wait: with overlap on, the
+ * kernel that immediately precedes decode_step must not write pool pages that this step reads,
+ * unless it is a decode_step itself (whose appended rows this step replaces in its staged tiles
+ * anyway).  Turning overlap off restores plain stream order.  Errors: CKV_EINVAL. */
 int32_t ckv_set_overlap(ckv_pool *pool, int32_t enable);
 
 /* Synchronise `stream`, read and clear the device status word.  Returns CKV_OK, CKV_EBOUNDS

@@ -18,7 +18,7 @@ LIBRARY = os.path.join(_HERE, "libchiron_kv.so")
 
 CKV_OK, CKV_EINVAL, CKV_ENOMEM, CKV_ECUDA, CKV_EBOUNDS, CKV_ETIMEOUT = 0, -1, -2, -3, -4, -5
 STATUS_BAD_LENGTH, STATUS_BAD_PAGE, STATUS_WAIT_LIMIT = 1, 2, 4
-PIECE_COST_TILES = 2                       # the plan's per-piece overhead units (TILE_TOKENS: set from the library below)
+TILE_TOKENS, PIECE_COST_TILES = 32, 2      # the plan's tile size and per-piece overhead units
 
 EXPORTS = (
     "kv_pool_bytes", "kv_workspace_bytes", "kv_pool_create", "kv_pool_destroy", "kv_append",
@@ -26,7 +26,7 @@ EXPORTS = (
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
     "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace", "ckv_set_overlap",
     "decode_attention_noalloc", "decode_step", "kv_swap_out", "kv_swap_in",
-    "kv_append_multi", "decode_attention_multi", "ckv_max_cells", "ckv_tile_tokens", "ckv_set_dynamic",
+    "kv_append_multi", "decode_attention_multi",
     "local_autoscaler_instance_slo", "local_autoscaler_create", "local_autoscaler_destroy",
     "local_autoscaler_update", "local_autoscaler_get", "local_autoscaler_simulate",
     "global_request_groups", "global_waiting_time", "global_batch_backpressure", "global_batch_autoscale",
@@ -74,9 +74,6 @@ def _load() -> ctypes.CDLL:
     lib.decode_plan.restype = i32; lib.decode_plan.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_set_partition.restype = i32; lib.ckv_set_partition.argtypes = [vp, i32]
     lib.ckv_set_overlap.restype = i32; lib.ckv_set_overlap.argtypes = [vp, i32]
-    lib.ckv_set_dynamic.restype = i32; lib.ckv_set_dynamic.argtypes = [vp, i32, i32, i32]
-    lib.ckv_max_cells.restype = i32; lib.ckv_max_cells.argtypes = []
-    lib.ckv_tile_tokens.restype = i32; lib.ckv_tile_tokens.argtypes = []
     lib.ckv_get_partition.restype = i32; lib.ckv_get_partition.argtypes = [vp]
     lib.kv_check_status.restype = i32; lib.kv_check_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.decode_step_host.restype = i32; lib.decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
@@ -111,7 +108,6 @@ def _load() -> ctypes.CDLL:
 
 
 lib = _load()
-TILE_TOKENS = int(lib.ckv_tile_tokens())     # tokens per tile, the plan's scheduling unit
 
 
 def last_error() -> str:
@@ -246,21 +242,14 @@ class KvPool:
                   image.numel() * image.element_size(), _stream_ptr(stream)))
 
     def decode_plan(self, seq_lens, stream=None):
-        """(header dict, int32 [num_cells][4] array of cell starts; the first num_spans cells are the spans)."""
+        """(header dict, int32 [num_spans][4] array of span starts)."""
         batch = int(seq_lens.shape[0])
-        header = np.zeros(16, dtype=np.int32)
-        starts = np.zeros((int(lib.ckv_max_cells()), 4), dtype=np.int32)
+        header = np.zeros(4, dtype=np.int32)
+        starts = np.zeros((self.get_partition(), 4), dtype=np.int32)
         _check(lib.decode_plan(self._h, batch, _dev_ptr(seq_lens, torch.int32), _stream_ptr(stream),
                                header.ctypes.data, starts.ctypes.data))
-        keys = ("total_units", "units_per_span", "num_spans", "spans_with_units", "num_cells")
-        hdr = dict(zip(keys, header[:5].tolist()))
-        hdr["dyn_cells"] = header[5:7].tolist()
-        hdr["dyn_pitch"] = header[7:9].tolist()
-        return hdr, starts[:hdr["num_cells"]].copy()
-
-    def set_dynamic(self, permille: int, cell_units_1: int = 8, cell_units_2: int = 3) -> None:
-        """Share (thousandths) of the work handed out dynamically and the two cell sizes (units)."""
-        _check(lib.ckv_set_dynamic(self._h, int(permille), int(cell_units_1), int(cell_units_2)))
+        keys = ("total_units", "units_per_span", "num_spans", "spans_with_units")
+        return dict(zip(keys, header.tolist())), starts
 
     def set_partition(self, num_spans: int) -> None:
         _check(lib.ckv_set_partition(self._h, int(num_spans)))

@@ -50,18 +50,6 @@ int32_t fail(int32_t code, const char *fmt, ...)
 constexpr int kWarps128 = CKV_WARPS128, kStages128 = CKV_STAGES128;   // head_dim 128: 4 warps x 3 stages x 16 KB = 192 KB per SM
 constexpr int kWarps64 = CKV_WARPS64, kStages64 = CKV_STAGES64;       // head_dim 64:  4 warps x 4 stages x 8 KB
 constexpr int kMaxProfile = 4096;
-// Default share (thousandths) of the plan's units that warps claim dynamically, and the sizes of
-// the two runs of dynamic cells (units).  0 keeps the partition static.
-#ifndef CKV_DYN_PERMILLE
-#define CKV_DYN_PERMILLE 0
-#endif
-#ifndef CKV_DYN_CELL1
-#define CKV_DYN_CELL1 8
-#endif
-#ifndef CKV_DYN_CELL2
-#define CKV_DYN_CELL2 3
-#endif
-constexpr int kDynPermille = CKV_DYN_PERMILLE, kDynCell1 = CKV_DYN_CELL1, kDynCell2 = CKV_DYN_CELL2;
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -90,7 +78,7 @@ bool config_ok(const ckv_config *c, const char **why)
 }
 
 struct WorkspaceLayout {
-    size_t status, header, span_start, part_acc, part_ml, arrivals, sched, trace;
+    size_t status, header, span_start, part_acc, part_ml, arrivals, trace;
     size_t st_tables, st_lens, st_q, st_k, st_v, st_out;
     size_t total;
 };
@@ -103,11 +91,10 @@ WorkspaceLayout carve(const ckv_config &c)
     const size_t d2 = (size_t)c.head_dim * 2;
     w.status = take(256);
     w.header = take(sizeof(ckv::PlanHeader));
-    w.span_start = take(sizeof(int4) * ckv::kMaxCells);
-    w.part_acc = take(sizeof(float) * 2 * ckv::kMaxCells * ckv::kMaxGroup * c.head_dim);
-    w.part_ml = take(sizeof(float) * 2 * ckv::kMaxCells * 2 * ckv::kMaxGroup);
-    w.arrivals = take(sizeof(int32_t) * ckv::kMaxCells);
-    w.sched = take(256);
+    w.span_start = take(sizeof(int4) * ckv::kMaxSpans);
+    w.part_acc = take(sizeof(float) * 2 * ckv::kMaxSpans * ckv::kMaxGroup * c.head_dim);
+    w.part_ml = take(sizeof(float) * 2 * ckv::kMaxSpans * 2 * ckv::kMaxGroup);
+    w.arrivals = take(sizeof(int32_t) * ckv::kMaxSpans);
     w.trace = take(sizeof(unsigned long long) * 8 * ckv::kMaxSpans);
     w.st_tables = take(sizeof(int32_t) * (size_t)c.max_batch * c.max_pages_per_req);
     w.st_lens = take(sizeof(int32_t) * (size_t)c.max_batch);
@@ -131,7 +118,6 @@ struct ckv_pool {
     int device;
     int num_sms;
     int num_spans;                   // partition width: one span per warp of the attention kernel
-    int dyn_permille, dyn_c1, dyn_c2; // share of the work handed out dynamically and the two cell sizes
     uint8_t *d_pool;
     uint8_t *d_ws;
     WorkspaceLayout ws;
@@ -195,10 +181,7 @@ int32_t launch_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, cu
     pp.max_pages_per_req = c.max_pages_per_req;
     pp.num_kv_heads = c.num_kv_heads;
     pp.num_spans = pool->num_spans;
-    pp.dyn_permille = pool->dyn_permille;
-    pp.dyn_c1 = pool->dyn_c1;
-    pp.dyn_c2 = pool->dyn_c2;
-    ckv::splitkv_plan_kernel<<<std::min((ckv::kMaxCells + 7) / 8, 4 * pool->num_sms), 256, 0, stream>>>(pp);
+    ckv::splitkv_plan_kernel<<<(pool->num_spans + 7) / 8, 256, 0, stream>>>(pp);
     CKV_CUDA(cudaGetLastError());
     pool->launches += 1;
     return CKV_OK;
@@ -210,7 +193,6 @@ int32_t launch_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, cu
 // ------------------------------------------------------------------------------------------
 constexpr int kNoAllocMaxSpans = 640;
 constexpr size_t kNaStatus = 0;                                                       // 256 B
-constexpr size_t kNaSched = 128;                                                      // int32 [2] inside the first 256 B
 constexpr size_t kNaArrivals = 256;                                                   // int32 [640]
 constexpr size_t kNaSpanStart = kNaArrivals + sizeof(int32_t) * kNoAllocMaxSpans;     // int4 [640]
 constexpr size_t kNaTrace = kNaSpanStart + sizeof(int4) * kNoAllocMaxSpans;           // u64 [640][8]
@@ -288,9 +270,6 @@ int32_t kv_pool_create(const ckv_config *cfg, void *d_pool, size_t pool_bytes, v
     p->d_pool = static_cast<uint8_t *>(d_pool);
     p->d_ws = static_cast<uint8_t *>(d_workspace);
     p->ws = ws;
-    p->dyn_permille = kDynPermille;
-    p->dyn_c1 = kDynCell1;
-    p->dyn_c2 = kDynCell2;
     p->launches = 0;
     p->profile = false;
     p->overlap = true;
@@ -439,10 +418,6 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
     ap.part_acc = pool->wsp<float>(pool->ws.part_acc);
     ap.part_ml = pool->wsp<float>(pool->ws.part_ml);
     ap.arrivals = pool->wsp<int32_t>(pool->ws.arrivals);
-    ap.sched = pool->wsp<int32_t>(pool->ws.sched);
-    ap.dyn_permille = pool->dyn_permille;
-    ap.dyn_c1 = pool->dyn_c1;
-    ap.dyn_c2 = pool->dyn_c2;
     ap.span_start = pool->wsp<int4>(pool->ws.span_start);
     ap.trace = pool->wsp<unsigned long long>(pool->ws.trace);
     ap.status = pool->wsp<uint32_t>(pool->ws.status);
@@ -516,26 +491,8 @@ int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, vo
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (int32_t rc = launch_plan(pool, batch, d_seq_lens, s)) return rc;
     CKV_CUDA(cudaMemcpyAsync(h_header, pool->d_ws + pool->ws.header, sizeof(ckv::PlanHeader), cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaMemcpyAsync(h_span_start, pool->d_ws + pool->ws.span_start, sizeof(int4) * pool->num_spans, cudaMemcpyDeviceToHost, s));
     CKV_CUDA(cudaStreamSynchronize(s));
-    const int32_t cells = reinterpret_cast<const ckv::PlanHeader *>(h_header)->num_cells;
-    if (cells < 0 || cells > ckv::kMaxCells) return fail(CKV_ECUDA, "decode_plan: the plan kernel reported %d cells", cells);
-    CKV_CUDA(cudaMemcpyAsync(h_span_start, pool->d_ws + pool->ws.span_start, sizeof(int4) * cells, cudaMemcpyDeviceToHost, s));
-    CKV_CUDA(cudaStreamSynchronize(s));
-    return CKV_OK;
-}
-
-int32_t ckv_max_cells(void) { return ckv::kMaxCells; }
-int32_t ckv_tile_tokens(void) { return ckv::kTileTokens; }
-
-int32_t ckv_set_dynamic(ckv_pool *pool, int32_t permille, int32_t cell_units_1, int32_t cell_units_2)
-{
-    if (!pool) return fail(CKV_EINVAL, "ckv_set_dynamic: pool is NULL");
-    if (permille < 0 || permille > 900) return fail(CKV_EINVAL, "ckv_set_dynamic: share %d outside [0, 900] thousandths", permille);
-    if (permille > 0 && (cell_units_1 < 1 || cell_units_2 < 0 || cell_units_2 > cell_units_1))
-        return fail(CKV_EINVAL, "ckv_set_dynamic: cell sizes must satisfy 1 <= first, 0 <= second <= first");
-    pool->dyn_permille = permille;
-    pool->dyn_c1 = cell_units_1;
-    pool->dyn_c2 = cell_units_2;
     return CKV_OK;
 }
 
@@ -550,8 +507,7 @@ int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits)
     if (out_bits) *out_bits = bits;
     if (bits & ckv::kStatusWaitLimit) {
         // a warp that gave up may have left arrival counters half-way; start the next launch clean
-        CKV_CUDA(cudaMemsetAsync(pool->d_ws + pool->ws.arrivals, 0, sizeof(int32_t) * ckv::kMaxCells, s));
-        CKV_CUDA(cudaMemsetAsync(pool->d_ws + pool->ws.sched, 0, 256, s));
+        CKV_CUDA(cudaMemsetAsync(pool->d_ws + pool->ws.arrivals, 0, sizeof(int32_t) * ckv::kMaxSpans, s));
         CKV_CUDA(cudaStreamSynchronize(s));
     }
     if (bits & ckv::kStatusWaitLimit) return fail(CKV_ETIMEOUT, "device status 0x%x: a bounded wait gave up", bits);
@@ -756,9 +712,6 @@ int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int3
     ap.part_acc = reinterpret_cast<float *>(scratch + kNaPartAcc);
     ap.part_ml = reinterpret_cast<float *>(scratch + kNaPartMl);
     ap.arrivals = reinterpret_cast<int32_t *>(scratch + kNaArrivals);
-    ap.sched = reinterpret_cast<int32_t *>(scratch + kNaSched);
-    ap.dyn_permille = 0;                          // static partition only: the scratch has one pair of slots per span
-    ap.dyn_c1 = ap.dyn_c2 = 0;
     ap.span_start = reinterpret_cast<int4 *>(scratch + kNaSpanStart);
     ap.trace = reinterpret_cast<unsigned long long *>(scratch + kNaTrace);
     ap.status = reinterpret_cast<uint32_t *>(scratch + kNaStatus);

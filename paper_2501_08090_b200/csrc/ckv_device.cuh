@@ -19,7 +19,6 @@ constexpr int kPagesPerTile = CKV_PAGES_PER_TILE;   // a tile is the scheduling 
 constexpr int kTileTokens = kPageSize * kPagesPerTile;
 constexpr int kMaxGroup = 8;         // query heads per KV head handled by one MMA column block
 constexpr int kMaxSpans = 2048;      // upper bound on the partition width (one span per warp)
-constexpr int kMaxCells = 6144;      // upper bound on spans plus dynamically claimed cells (partial slots, counters)
 constexpr int kMaxBatch = 8192;
 constexpr int kBulkMergeFrom = 4;    // merges of more partials than this go through shared memory
 constexpr int kTreeFrom = 12;        // pairs cut into more partials than this are merged in two levels
@@ -53,74 +52,7 @@ struct PlanHeader {
     int32_t units_per_span;
     int32_t num_spans;
     int32_t spans_with_units;
-    int32_t num_cells;               // spans + dynamically claimed cells
-    int32_t dyn_cells[2], dyn_pitch[2];
-    int32_t reserved[7];
 };
-
-// The cells of the partition.  The unit axis is cut into num_spans "static" cells of q0 units,
-// one per warp, which every warp starts on without asking anybody, followed -- when a share of
-// the work is set aside for balancing -- by two runs of smaller cells (n1 of c1 units, then n2 of
-// c2 <= c1 units) that warps claim from a counter as they become free: SMs do not all stream at
-// the same rate, so the faster ones take more of these.  Cell indices grow with the unit index,
-// so the cells that hold tiles of one (request, kv head) are consecutive.  With no dynamic share
-// this is the plain partition: span s owns units [s*q0, (s+1)*q0).
-struct CellGrid {
-    long long total;                 // units on the axis
-    long long s0, s1;                // first unit of the first and of the second dynamic run
-    int n0, q0, n1, c1, n2, c2;
-
-    __host__ __device__ __forceinline__ int cells() const { return n0 + n1 + n2; }
-    __host__ __device__ __forceinline__ int cell_of(long long u) const
-    {
-        if (u < s0) return (int)(u / q0);
-        if (u < s1) return n0 + (int)((u - s0) / c1);
-        return n0 + n1 + (int)((u - s1) / c2);
-    }
-    __host__ __device__ __forceinline__ long long begin_of(int k) const
-    {
-        if (k < n0) return (long long)k * q0 < s0 ? (long long)k * q0 : s0;
-        if (k < n0 + n1) return s0 + (long long)(k - n0) * c1;
-        const long long b = s1 + (long long)(k - n0 - n1) * c2;
-        return b < total ? b : total;
-    }
-    __host__ __device__ __forceinline__ long long end_of(int k) const
-    {
-        if (k < n0) { const long long e = (long long)(k + 1) * q0; return e < s0 ? e : s0; }
-        if (k < n0 + n1) { const long long e = s0 + (long long)(k - n0 + 1) * c1; return e < s1 ? e : s1; }
-        const long long e = s1 + (long long)(k - n0 - n1 + 1) * c2;
-        return e < total ? e : total;
-    }
-};
-
-// dyn_permille: thousandths of the units set aside for the dynamic cells (0: none); c1, c2: their
-// sizes.  Small problems (fewer than 8 units per span) stay static.  If the dynamic cells would
-// exceed the slots there are, their sizes are doubled until they fit.
-__host__ __device__ __forceinline__ CellGrid make_cell_grid(long long total, int num_spans, int dyn_permille, int c1, int c2)
-{
-    CellGrid g;
-    g.total = total; g.n0 = num_spans; g.n1 = g.n2 = 0;
-    g.c1 = c1 > 0 ? c1 : 1; g.c2 = c2 > 0 ? c2 : 1;
-    long long dyn = 0;
-    if (dyn_permille > 0 && c1 > 0 && total >= 8ll * num_spans) dyn = total * dyn_permille / 1000;
-    const long long q = (total - dyn + num_spans - 1) / num_spans;
-    g.q0 = q > 1 ? (int)q : 1;
-    g.s0 = (long long)g.n0 * g.q0 < total ? (long long)g.n0 * g.q0 : total;
-    g.s1 = total;
-    const long long rest = total - g.s0;
-    if (rest > 0) {
-        const long long lvl1 = c2 > 0 ? rest * 2 / 3 : rest;
-        const int budget = kMaxCells - num_spans;
-        for (;;) {
-            const long long n1 = (lvl1 + g.c1 - 1) / g.c1;
-            const long long s1 = g.s0 + n1 * g.c1 < total ? g.s0 + n1 * g.c1 : total;
-            const long long n2 = (total - s1 + g.c2 - 1) / g.c2;
-            if (n1 + n2 <= budget) { g.n1 = (int)n1; g.n2 = (int)n2; g.s1 = s1; break; }
-            g.c1 *= 2; g.c2 *= 2;
-        }
-    }
-    return g;
-}
 
 // A context length is usable if min_len <= L <= table capacity (min_len = the number of new
 // tokens of the step, 1 for plain decode); otherwise the request has no tiles.
@@ -245,7 +177,8 @@ struct SpanStart {
     int tiles_r;           // tiles per kv head of request r
     int L;                 // context length of request r
     long long v;           // unit index of that first tile
-    long long end;         // one past the cell's last unit
+    long long end;         // one past the span's last unit
+    int total, q;          // header values
 };
 
 // Requests with an unusable length get their output rows cleared and the status word flagged.
@@ -271,31 +204,26 @@ __device__ __forceinline__ void flag_unusable_requests(const int32_t *__restrict
 // Units of one kv head of a request with t tiles (0 if the request is unusable).
 __device__ __forceinline__ int units_of_tiles(int t) { return t > 0 ? t + kPieceCostTiles : 0; }
 
-// Executed by one whole warp: the number of units on the plan's axis.
-__device__ __forceinline__ long long warp_total_units(const int32_t *__restrict__ seq_lens, int batch, int max_pages_per_req,
-                                                      int num_kv_heads, int lane, int min_len = 1)
+// Executed by one whole warp.  Two passes over seq_lens: the total number of units, then the
+// (request, kv head) that holds unit span*q and the first tile at or after it.
+__device__ __forceinline__ SpanStart warp_plan(const int32_t *__restrict__ seq_lens, int batch, int max_pages_per_req,
+                                               int num_kv_heads, int num_spans, int span, int lane, int min_len = 1)
 {
-    long long sum = 0;
+    SpanStart s;
+    int sum = 0;
     for (int base = 0; base < batch; base += 32) {
         const int r = base + lane;
         if (r < batch) sum += units_of_tiles(tiles_of_length(__ldg(seq_lens + r), max_pages_per_req, min_len));
     }
 #pragma unroll
     for (int x = 16; x > 0; x >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, x);
-    return sum * num_kv_heads;
-}
-
-// Executed by one whole warp: the (request, kv head) that holds unit `begin` and the first tile at
-// or after it, for the cell [begin, end) of an axis of `total` units.  r = -1 if the cell holds no tile.
-__device__ __forceinline__ SpanStart warp_locate(const int32_t *__restrict__ seq_lens, int batch, int max_pages_per_req,
-                                                 int num_kv_heads, long long total, long long begin, long long end,
-                                                 int lane, int min_len = 1)
-{
-    SpanStart s;
+    s.total = sum * num_kv_heads;
+    s.q = max(1, (s.total + num_spans - 1) / num_spans);
+    const long long begin = (long long)span * s.q;
     s.r = -1; s.h = s.tile = s.tiles_r = s.L = 0;
-    s.v = s.end = min(begin, total);
-    if (begin >= total || begin >= end) return s;
-    s.end = min(end, total);
+    s.v = s.end = min(begin, (long long)s.total);
+    if (begin >= s.total) return s;
+    s.end = min(begin + s.q, (long long)s.total);
 
     long long running = 0;                               // units (all heads) before request `base`
     for (int base = 0; base < batch; base += 32) {
@@ -318,9 +246,9 @@ __device__ __forceinline__ SpanStart warp_locate(const int32_t *__restrict__ seq
             const long long before = __shfl_sync(0xffffffffu, upto, src) - (long long)u_r * num_kv_heads;
             const int rem = (int)(begin - before);
             const int h = rem / u_r, off = rem % u_r;
-            const int tile = max(0, off - kPieceCostTiles);               // a cell starting in the overhead
+            const int tile = max(0, off - kPieceCostTiles);               // a span starting in the overhead
             const long long v = before + (long long)h * u_r + kPieceCostTiles + tile;   // units starts at tile 0
-            if (v >= s.end) return s;                                      // the cell holds overhead units only
+            if (v >= s.end) return s;                                      // the span holds overhead units only
             s.r = base + src; s.tiles_r = t_r; s.L = L_r;
             s.h = h; s.tile = tile; s.v = v;
             return s;
@@ -333,30 +261,23 @@ __device__ __forceinline__ SpanStart warp_locate(const int32_t *__restrict__ seq
 struct PlanParams {
     const int32_t *seq_lens;
     PlanHeader *header;
-    int4 *span_start;               // [cells] request, kv head, tile, unit index of that tile (-1s if empty)
+    int4 *span_start;               // [num_spans] request, kv head, tile, unit index of that tile (-1s if idle)
     int32_t batch, max_pages_per_req, num_kv_heads, num_spans;
-    int32_t dyn_permille, dyn_c1, dyn_c2;
 };
 
 __global__ void splitkv_plan_kernel(const PlanParams p)
 {
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
-    const long long total = warp_total_units(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, lane);
-    const CellGrid g = make_cell_grid(total, p.num_spans, p.dyn_permille, p.dyn_c1, p.dyn_c2);
-    for (int cell = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; cell < g.cells(); cell += warps) {
-        const SpanStart s = warp_locate(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, total,
-                                        g.begin_of(cell), g.end_of(cell), lane);
+    for (int span = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; span < p.num_spans; span += warps) {
+        const SpanStart s = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane);
         if (lane == 0) {
-            p.span_start[cell] = s.r < 0 ? make_int4(-1, -1, -1, -1) : make_int4(s.r, s.h, s.tile, (int)s.v);
-            if (cell == 0) {
-                p.header->total_units = (int)total;
-                p.header->units_per_span = g.q0;
+            p.span_start[span] = s.r < 0 ? make_int4(-1, -1, -1, -1) : make_int4(s.r, s.h, s.tile, (int)s.v);
+            if (span == 0) {
+                p.header->total_units = s.total;
+                p.header->units_per_span = s.q;
                 p.header->num_spans = p.num_spans;
-                p.header->spans_with_units = (int)((g.s0 + g.q0 - 1) / g.q0);
-                p.header->num_cells = g.cells();
-                p.header->dyn_cells[0] = g.n1; p.header->dyn_cells[1] = g.n2;
-                p.header->dyn_pitch[0] = g.c1; p.header->dyn_pitch[1] = g.c2;
+                p.header->spans_with_units = (s.total + s.q - 1) / s.q;
             }
         }
     }
@@ -550,10 +471,9 @@ struct AttnParams {
     const uint4 *k_new;             // bf16 [batch][Hkv][d]
     const uint4 *v_new;
     uint4 *pool_layer;
-    float *part_acc;                // [2*kMaxCells][8][D]
-    float *part_ml;                 // [2*kMaxCells][16]  (m[8], l[8])
-    int32_t *arrivals;              // [kMaxCells], all zero between launches
-    int32_t *sched;                 // [0] next dynamic cell to hand out, [1] warps that have left; zero between launches
+    float *part_acc;                // [2*kMaxSpans][8][D]
+    float *part_ml;                 // [2*kMaxSpans][16]  (m[8], l[8])
+    int32_t *arrivals;              // [kMaxSpans], all zero between launches
     int4 *span_start;               // [kMaxSpans] what each span started at (diagnostic)
     unsigned long long *trace;      // [kMaxSpans][8] ns: start, first tile landed, last tile done, span done,
                                     //   total wait for data, total time between pieces, tiles, pieces
@@ -561,7 +481,6 @@ struct AttnParams {
     int32_t batch, max_pages_per_req, num_pages, num_kv_heads, num_q_heads, group;
     int32_t layer_page_base;        // layer * num_pages
     int32_t num_spans;
-    int32_t dyn_permille, dyn_c1, dyn_c2;   // share and sizes of the dynamically claimed cells (make_cell_grid)
     int32_t q_len;                  // new tokens per request in this step (1 for plain decode); q_len*group <= 8
     float scale_log2;               // log2(e) / sqrt(d)
 };
@@ -846,7 +765,7 @@ struct AttnLayout {
     static constexpr int kStagePitch = D + 4;                    // floats per staging row (bank spread)
     static constexpr int kStagingBytes = kMaxGroup * kStagePitch * 4;
     static constexpr int kRingBytes = W * NS * kStageBytes;
-    static constexpr int kSmemBytes = kRingBytes + W * kStagingBytes + W * (NS + 1) * 8 + 1024;   // + one merge barrier per warp
+    static constexpr int kSmemBytes = kRingBytes + W * kStagingBytes + W * NS * 8 + 1024;
     static constexpr int kThreads = W * 32;
 };
 
@@ -888,8 +807,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 
     const uint32_t ring = smem_u32(smem) + warp * NS * Lay::kStageBytes;
     float *staging = (float *)(smem + Lay::kRingBytes + warp * Lay::kStagingBytes);
-    const uint32_t bars = smem_u32(smem + Lay::kRingBytes + W * Lay::kStagingBytes) + warp * (NS + 1) * 8;
-    const uint32_t merge_bar = bars + NS * 8;    // used by merges that stage partials in the idle ring
+    const uint32_t bars = smem_u32(smem + Lay::kRingBytes + W * Lay::kStagingBytes) + warp * NS * 8;
 
     grid_launch_dependents();
     if (span >= p.num_spans) return;
@@ -897,29 +815,24 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     if (lane == 0) {
         t_start = global_timer_ns();
         prefetch_tensormap(&tmap);
-        for (int s = 0; s <= NS; ++s) mbar_init(bars + s * 8, 1);
+        for (int s = 0; s < NS; ++s) mbar_init(bars + s * 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
     __syncwarp();
 
-    // ---- plan: the cells of this launch.  This warp starts on cell `span`; when dynamic cells
-    // exist it claims more of them, one at a time, until none is left.
+    // ---- plan: where does this warp's span start?
     // Nothing read up to the dependency wait below is written by the preceding kernel of a decode
     // step (the KV append writes only the pool), so this prologue overlaps that kernel's tail.
-    const long long total_units = warp_total_units(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, lane, p.q_len);
-    const CellGrid grid = make_cell_grid(total_units, p.num_spans, p.dyn_permille, p.dyn_c1, p.dyn_c2);
-    const int n_dyn = grid.n1 + grid.n2;
-    int cell = span;
-    SpanStart st = warp_locate(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, total_units,
-                               grid.begin_of(cell), grid.end_of(cell), lane, p.q_len);
+    const SpanStart st = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane,
+                                   p.q_len);
     if (st.r < 0 || span == 0) {
         grid_dependency_wait();
         if (span == 0)
             flag_unusable_requests(p.seq_lens, p.batch, p.max_pages_per_req, p.q_len, lane, p.out,
                                    p.q_len * p.num_q_heads * D, p.status);
     }
-    if (st.r < 0 && n_dyn == 0) {
+    if (st.r < 0) {
         if (lane == 0) {
             p.span_start[span] = make_int4(-1, -1, -1, -1);
             p.trace[span * 8 + 0] = t_start;
@@ -928,16 +841,17 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         if (lane == 0) p.trace[span * 8 + 2] = p.trace[span * 8 + 3] = global_timer_ns();
         return;
     }
-    long long v_end = st.end;
+    const long long v_end = st.end;
+    const int q_span = st.q;
     const int G = p.group;
     const int ncols = G * p.q_len;               // live MMA columns: column c = new token c / G, head c % G
     const int qi_stride = p.num_q_heads * D;     // elements between a request's consecutive new tokens in q / out
 
     // ---- issue side: block-table entries travel in registers, 32 pages (16 tiles) per chunk
     SpanCursor ic;
-    ic.r = ic.h = ic.tile = ic.L = ic.tiles = 0; ic.v = 0;
-    bool more_to_issue = false;                  // the issue cursor still points at a tile of the current cell
-    int issued = 0;                              // tiles issued so far, over all cells: stage and phase follow from it
+    ic.r = st.r; ic.h = st.h; ic.tile = st.tile; ic.L = st.L; ic.tiles = st.tiles_r; ic.v = st.v;
+    bool more_to_issue = true;                   // the issue cursor still points at a tile of this span
+    int issued = 0;
     bool alive = true;
     auto table_row = [&](int r) { return p.block_tables + (size_t)r * p.max_pages_per_req; };
     auto load_chunk = [&](int r, int chunk) -> int {
@@ -945,9 +859,12 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         return (r < p.batch && idx < p.max_pages_per_req) ? __ldg(table_row(r) + idx) : -1;
     };
     constexpr int kTilesPerChunk = 32 / kPagesPerTile;
-    int cur_chunk = 0, cur_val = -1, nxt_val = -1;
+    int cur_chunk = ic.tile / kTilesPerChunk;
+    int cur_val = load_chunk(ic.r, cur_chunk);
+    int nxt_val = load_chunk(ic.r, cur_chunk + 1);
     // chunk 0 of the row the NEXT (request, kv head) will read: this row again, or the next request's
-    int pf_row = 0, pf_val = -1;
+    int pf_row = (ic.h + 1 < p.num_kv_heads) ? ic.r : ic.r + 1;
+    int pf_val = load_chunk(pf_row, 0);
 
     // query fragments of a (request, kv head), fetched when the issue cursor enters it
     uint32_t qn[Lay::kKSteps][2];
@@ -977,6 +894,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 #ifdef CKV_TRACE_WAITS
     unsigned long long t_issue = 0, t_masked = 0;
 #endif
+    bool inputs_ready = true;                    // q, k_new and v_new may be read (the dependency wait is behind us)
     auto issue_next = [&]() {
 #ifdef CKV_TRACE_WAITS
         const unsigned long long i0 = global_timer_ns();
@@ -1006,7 +924,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             tma_load_2d(ring + slot * Lay::kStageBytes + pg * Lay::kPageBytes + hf * Lay::kHalfBytes,
                         &tmap, hf * 64, y, bars + slot * 8);
         }
-        if (p.k_new != nullptr && ic.tile == ic.tiles - 1 && an_r < 0) {
+        if (p.k_new != nullptr && ic.tile == ic.tiles - 1 && an_r < 0 && inputs_ready) {
             // last tile of this (request, kv head): fetch the rows to append and remember their page
             const bool bad = page < 0 || page >= p.num_pages;               // before any redirect above
             an_val = load_new_rows(ic.r, ic.h);
@@ -1023,7 +941,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 nxt_val = load_chunk(ic.r, 1);
                 pf_row = (ic.h + 1 < p.num_kv_heads) ? ic.r : ic.r + 1;
                 pf_val = (pf_row == ic.r) ? cur_val : load_chunk(pf_row, 0);
-                if (qn_r < 0) {
+                if (qn_r < 0 && inputs_ready) {
                     load_q(qn, ic.r, ic.h);
                     qn_r = ic.r; qn_h = ic.h;
                 }
@@ -1034,20 +952,28 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 #endif
     };
 
-    // Point the issue cursor at the first tile of the cell that `st` describes.
-    auto enter_cell = [&]() {
-        ic.r = st.r; ic.h = st.h; ic.tile = st.tile; ic.L = st.L; ic.tiles = st.tiles_r; ic.v = st.v;
-        more_to_issue = true;
-        cur_chunk = ic.tile / kTilesPerChunk;
-        cur_val = load_chunk(ic.r, cur_chunk);
-        nxt_val = load_chunk(ic.r, cur_chunk + 1);
-        pf_row = (ic.h + 1 < p.num_kv_heads) ? ic.r : ic.r + 1;
-        pf_val = load_chunk(pf_row, 0);
-        qn_r = -1; an_r = -1;
-    };
+    // A step with the fused append is the only writer of its layer's pool, and what it computes does
+    // not depend on whether a tile's copy saw this step's new rows (they are put into the staged
+    // tile before use).  Its first loads can therefore start before the preceding kernel has
+    // finished -- under that kernel's tail -- as long as nothing of q, k_new or v_new is touched yet.
+    const bool early = p.k_new != nullptr;
+    if (early) {
+        inputs_ready = false;
+        for (int k = 0; k < NS && more_to_issue; ++k) issue_next();
+        inputs_ready = true;
+    }
+    grid_dependency_wait();                       // the workspace, q, the new rows and `out` are ours from here on
+    if (lane == 0) {
+        p.span_start[span] = make_int4(st.r, st.h, st.tile, (int)st.v);
+        p.trace[span * 8 + 0] = t_start;
+        p.trace[span * 8 + 1] = 0;
+    }
+    if (!early)
+        for (int k = 0; k < NS && more_to_issue; ++k) issue_next();
 
     // ---- compute side
     SpanCursor cc;
+    cc.r = st.r; cc.h = st.h; cc.tile = st.tile; cc.L = st.L; cc.tiles = st.tiles_r; cc.v = st.v;
     const int g0 = (lane & 3) * 2;               // first of the two group columns this lane accumulates
     const int qi0 = g0 / G, qi1 = (g0 + 1) / G;  // the new tokens those two columns belong to
     uint32_t k_off[4], v_off[4];                 // ldmatrix lane offsets inside one page block
@@ -1063,33 +989,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         }
     }
 
-    int done = 0;                                // tiles computed (or skipped after a wait gave up), over all cells
+    int done = 0;                                // tiles computed (or skipped after a wait gave up)
     int landed = 0;                              // tiles whose copies were seen to complete
-    unsigned long long t_wait = 0, t_between = 0, t_piece_end = 0;
-    int n_pieces = 0, n_cells = 0;
-    int merge_uses = 0;                          // phases the merge barrier has completed
-    bool waited = (st.r < 0 || span == 0);       // the dependency wait has been executed
-    for (;;) {                                   // one pass per cell
-    if (st.r >= 0) enter_cell();                 // table reads only: inputs, not written by the preceding kernel
-    if (!waited) {
-        grid_dependency_wait();                  // the pool, the workspace and `out` are ours from here on
-        waited = true;
-    }
-    if (n_cells == 0 && lane == 0) {
-        p.span_start[span] = st.r < 0 ? make_int4(-1, -1, -1, -1) : make_int4(st.r, st.h, st.tile, (int)st.v);
-        p.trace[span * 8 + 0] = t_start;
-        p.trace[span * 8 + 1] = 0;
-    }
-    // claim the next cell now; the answer is needed only when this cell has been streamed
-    int ticket = 0x7fffffff;
-    if (n_dyn > 0 && lane == 0) ticket = atomicAdd(p.sched, 1);
-    if (st.r >= 0) {
-    ++n_cells;
-    for (int k = 0; k < NS && more_to_issue; ++k) issue_next();
-    cc.r = st.r; cc.h = st.h; cc.tile = st.tile; cc.L = st.L; cc.tiles = st.tiles_r; cc.v = st.v;
     bool more_to_compute = true;
+    unsigned long long t_wait = 0, t_between = 0, t_piece_end = 0;
+    int n_pieces = 0;
     bool first_piece = true;
-    // a cell writes at most two partials: its first piece and its last piece
+    // a span writes at most two partials: its first piece and its last piece
     int pend_first[2] = {-1, -1}, pend_last[2] = {0, 0}, pend_slot[2] = {0, 0};
     uint16_t *pend_out[2] = {nullptr, nullptr};
     while (more_to_compute) {
@@ -1128,7 +1034,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             const unsigned long long w1 = global_timer_ns();
 #endif
             ++landed;
-            if (landed == 1 && lane == 0) p.trace[span * 8 + 1] = global_timer_ns();
+            if (done == 0 && lane == 0) p.trace[span * 8 + 1] = global_timer_ns();
 
             const int ntok = min(kTileTokens, piece_L - ti * kTileTokens);      // tokens of the context in this tile
             // Causality among the step's new tokens: column c (new token c / G) sees the context up to
@@ -1294,11 +1200,11 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 }
             }
         } else {
-            const int slot_id = 2 * cell + (first_piece ? 0 : 1);
+            const int slot_id = 2 * span + (first_piece ? 0 : 1);
             float *pa = p.part_acc + (size_t)slot_id * kMaxGroup * D;
 #pragma unroll
             for (int g = 0; g < kMaxGroup; ++g)
-                if (lane * 4 < D)
+                if (g < ncols && lane * 4 < D)              // only the live columns are ever read back
                     *(float4 *)(pa + g * D + lane * 4) = *(const float4 *)(staging + g * Lay::kStagePitch + lane * 4);
             if (lane < 4) {
                 float *ml = p.part_ml + slot_id * 2 * kMaxGroup;
@@ -1309,12 +1215,12 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             // neither the fence nor a merge ever interrupts this warp's loads
             const long long tile0_unit = cc.v - piece_tile0;             // unit of this (request, kv head)'s tile 0
             const int k = first_piece ? 0 : 1;
-            pend_first[k] = grid.cell_of(tile0_unit);
-            pend_last[k] = grid.cell_of(tile0_unit + piece_tiles - 1);
-            // in cell pend_first the piece is that cell's first one iff the cell starts inside this
+            pend_first[k] = (int)(tile0_unit / q_span);
+            pend_last[k] = (int)((tile0_unit + piece_tiles - 1) / q_span);
+            // in span pend_first the piece is that span's first one iff the span starts inside this
             // (request, kv head)'s overhead units or exactly at them
-            pend_slot[k] = (grid.begin_of(pend_first[k]) >= tile0_unit - kPieceCostTiles) ? 2 * pend_first[k]
-                                                                                          : 2 * pend_first[k] + 1;
+            pend_slot[k] = ((long long)pend_first[k] * q_span >= tile0_unit - kPieceCostTiles) ? 2 * pend_first[k]
+                                                                                              : 2 * pend_first[k] + 1;
             pend_out[k] = out_rows;
         }
         __syncwarp();                             // staging is reused by the next piece
@@ -1343,7 +1249,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             sub[k] = 0; grp[k] = 0; grp_cnt[k] = n_part[k]; n_grp[k] = 1;
             if (n_part[k] > kTreeFrom) {
                 sub[k] = merge_group_size(n_part[k]);
-                grp[k] = (cell - pend_first[k]) / sub[k];
+                grp[k] = (span - pend_first[k]) / sub[k];
                 n_grp[k] = (n_part[k] + sub[k] - 1) / sub[k];
                 grp_cnt[k] = min(sub[k], n_part[k] - grp[k] * sub[k]);
             }
@@ -1366,12 +1272,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 if (last[0]) p.arrivals[pend_first[0] + (sub[0] ? 1 + grp[0] : 0)] = 0;
                 if (last[1]) p.arrivals[pend_first[1] + (sub[1] ? 1 + grp[1] : 0)] = 0;
             }
-            // the ring is idle now: every tile issued so far has been computed on
+            // stage 0's barrier has completed one phase per tile it carried; the ring is idle now
+            int bar_uses = (done + NS - 1) / NS;
             auto merge = [&](int k, const MergeSel sel, float *dst_acc, float *dst_ml) {
                 if (alive && sel.pieces > kBulkMergeFrom) {
                     fence_proxy_async();          // partials written through the generic proxy, read by bulk copies
                     alive = combine_partials_bulk<D>(p.part_acc, p.part_ml, pend_out[k], sel, dst_acc, dst_ml, ncols, G,
-                                                     qi_stride, lane, ring, NS * Lay::kStageBytes, merge_bar, merge_uses, p.status);
+                                                     qi_stride, lane, ring, NS * Lay::kStageBytes, bars, bar_uses, p.status);
                 } else {
                     combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], sel, dst_acc, dst_ml, ncols, G, qi_stride, lane);
                 }
@@ -1417,30 +1324,10 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             }
         }
     }
-    }   // the cell held tiles
-
-    // ---- the next cell, if dynamic cells exist and one is left
-    if (n_dyn == 0 || !alive) break;
-    ticket = __shfl_sync(0xffffffffu, ticket, 0);
-    if (ticket >= n_dyn) break;
-    cell = grid.n0 + ticket;
-    st = warp_locate(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, total_units,
-                     grid.begin_of(cell), grid.end_of(cell), lane, p.q_len);
-    v_end = st.end;
-    }   // one pass per cell
 
     // Do not leave while copies into this warp's ring may still be in flight (only after a wait gave up).
     if (!alive) {
         for (int k = landed; k < issued; ++k) mbar_wait_bounded(bars + (k % NS) * 8, (k / NS) & 1, p.status);
-    }
-    if (n_dyn > 0) {
-        // The last warp to leave puts the cell counter back to zero for the next launch.  Every
-        // warp's claims precede its own exit count, so none can follow the reset.
-        __threadfence();
-        if (lane == 0 && atomicAdd(p.sched + 1, 1) == min(p.num_spans, (int)(gridDim.x * W)) - 1) {
-            p.sched[0] = 0;
-            p.sched[1] = 0;
-        }
     }
     if (lane == 0) {
         p.trace[span * 8 + 3] = global_timer_ns();
@@ -1455,7 +1342,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         p.trace[span * 8 + 7] = t_masked;
 #else
         p.trace[span * 8 + 6] = done;
-        p.trace[span * 8 + 7] = (unsigned long long)n_pieces | ((unsigned long long)n_cells << 32);
+        p.trace[span * 8 + 7] = n_pieces;
 #endif
     }
 }

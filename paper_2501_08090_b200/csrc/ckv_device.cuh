@@ -763,9 +763,14 @@ struct AttnLayout {
     static constexpr int kKSteps = D / 16;
     static constexpr int kDTiles = D / 16;
     static constexpr int kStagePitch = D + 4;                    // floats per staging row (bank spread)
-    static constexpr int kStagingBytes = kMaxGroup * kStagePitch * 4;
+    static constexpr int kStagingBytes = (kMaxGroup * kStagePitch + 2 * kMaxGroup) * 4;   // rows, then m[8], l[8]
+    static constexpr int kParkBytes = (kMaxGroup * D + 2 * kMaxGroup) * 4;                // the same, rows unpadded
     static constexpr int kRingBytes = W * NS * kStageBytes;
-    static constexpr int kSmemBytes = kRingBytes + W * kStagingBytes + W * NS * 8 + 1024;
+    static constexpr int kStagingOff = kRingBytes;
+    static constexpr int kParkOff = kStagingOff + W * kStagingBytes;
+    static constexpr int kBarOff = kParkOff + W * kParkBytes;
+    static constexpr int kCtrOff = kBarOff + W * NS * 8;                                  // W counters of the CTA stage
+    static constexpr int kSmemBytes = kCtrOff + W * 4 + 1024;
     static constexpr int kThreads = W * 32;
 };
 
@@ -806,10 +811,14 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     const int span = blockIdx.x * W + warp;
 
     const uint32_t ring = smem_u32(smem) + warp * NS * Lay::kStageBytes;
-    float *staging = (float *)(smem + Lay::kRingBytes + warp * Lay::kStagingBytes);
-    const uint32_t bars = smem_u32(smem + Lay::kRingBytes + W * Lay::kStagingBytes) + warp * NS * 8;
+    float *staging = (float *)(smem + Lay::kStagingOff + warp * Lay::kStagingBytes);
+    float *park = (float *)(smem + Lay::kParkOff + warp * Lay::kParkBytes);
+    const uint32_t bars = smem_u32(smem + Lay::kBarOff) + warp * NS * 8;
+    int *cta_ctr = (int *)(smem + Lay::kCtrOff);
 
     grid_launch_dependents();
+    if (threadIdx.x < W) cta_ctr[threadIdx.x] = 0;
+    __syncthreads();                             // the only CTA-wide barrier: the counters of the CTA stage are zero
     if (span >= p.num_spans) return;
     unsigned long long t_start = 0;
     if (lane == 0) {
@@ -1200,27 +1209,28 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 }
             }
         } else {
-            const int slot_id = 2 * span + (first_piece ? 0 : 1);
-            float *pa = p.part_acc + (size_t)slot_id * kMaxGroup * D;
+            // The partial stays in shared memory until the span has been streamed.  A piece whose
+            // (request, kv head) began in an earlier span is this span's first piece: it moves to the
+            // parking buffer, since the staging tile is reused.  A piece whose pair begins here and
+            // runs on into the next span is the span's last piece and stays in the staging tile.
+            const bool entered = piece_tile0 > 0;
+            float *dst_ml = entered ? park + kMaxGroup * D : staging + kMaxGroup * Lay::kStagePitch;
+            if (entered) {
 #pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g)
-                if (g < ncols && lane * 4 < D)              // only the live columns are ever read back
-                    *(float4 *)(pa + g * D + lane * 4) = *(const float4 *)(staging + g * Lay::kStagePitch + lane * 4);
-            if (lane < 4) {
-                float *ml = p.part_ml + slot_id * 2 * kMaxGroup;
-                ml[g0] = m0; ml[g0 + 1] = m1;
-                ml[kMaxGroup + g0] = l0; ml[kMaxGroup + g0 + 1] = l1;
+                for (int g = 0; g < kMaxGroup; ++g)
+                    if (g < ncols && lane * 4 < D)
+                        *(float4 *)(park + g * D + lane * 4) = *(const float4 *)(staging + g * Lay::kStagePitch + lane * 4);
             }
-            // ---- remember the arrival; it is made once the whole span has been streamed, so that
-            // neither the fence nor a merge ever interrupts this warp's loads
+            if (lane < 4) {
+                dst_ml[g0] = m0; dst_ml[g0 + 1] = m1;
+                dst_ml[kMaxGroup + g0] = l0; dst_ml[kMaxGroup + g0 + 1] = l1;
+            }
+            // ---- remember the piece; it is handed on once the whole span has been streamed, so that
+            // neither a fence nor a merge ever interrupts this warp's loads
             const long long tile0_unit = cc.v - piece_tile0;             // unit of this (request, kv head)'s tile 0
-            const int k = first_piece ? 0 : 1;
-            pend_first[k] = (int)(tile0_unit / q_span);
+            const int k = entered ? 0 : 1;
+            pend_first[k] = (int)(tile0_unit / q_span);                   // first and last span that hold its tiles
             pend_last[k] = (int)((tile0_unit + piece_tiles - 1) / q_span);
-            // in span pend_first the piece is that span's first one iff the span starts inside this
-            // (request, kv head)'s overhead units or exactly at them
-            pend_slot[k] = ((long long)pend_first[k] * q_span >= tile0_unit - kPieceCostTiles) ? 2 * pend_first[k]
-                                                                                              : 2 * pend_first[k] + 1;
             pend_out[k] = out_rows;
         }
         __syncwarp();                             // staging is reused by the next piece
@@ -1234,13 +1244,78 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 
     if (lane == 0) p.trace[span * 8 + 2] = global_timer_ns();
 
-    // ---- arrivals: whichever warp arrives last for a (request, kv head) merges its partials (wait-free).
-    // A pair cut into more than kTreeFrom partials is merged in two levels: its partials form groups
-    // of `sub` consecutive ones, each with a counter of its own (kept in arrivals[] at the pair's
-    // interior spans, which no other pair uses); the last arriver of a group folds it into the slot
-    // of the group's first partial and then arrives for the pair, and the last group to arrive folds
-    // the group results.  Groups complete while other warps are still streaming, so the tail of the
-    // launch holds one short merge instead of one long one.
+    // ---- CTA stage.  Consecutive spans belong to the warps of one CTA, so the partials of a
+    // (request, kv head) that several of this CTA's warps hold are merged through shared memory:
+    // each warp counts itself in on a shared counter once its span has been streamed, and the last
+    // one folds the CTA's partials (wait-free, no global round trip).  If the pair lies inside this
+    // CTA the result is final; otherwise it is the CTA's one partial of the pair for the grid stage.
+    {
+        const int b0 = blockIdx.x * W;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            if (pend_first[k] < 0) continue;
+            const int f = pend_first[k], l = pend_last[k];
+            const int fb = max(f, b0), lb = min(l, b0 + W - 1), cb = lb - fb + 1;
+            pend_first[k] = -1;                   // becomes a grid-stage entry below, if one is needed
+            if (cb > 1) {
+                __threadfence_block();
+                __syncwarp();
+                int prior = 0;
+                if (lane == 0) prior = atomicAdd(cta_ctr + (fb - b0), 1);
+                prior = __shfl_sync(0xffffffffu, prior, 0);
+                if (prior != cb - 1) continue;    // a later warp of this CTA folds them
+                __threadfence_block();
+            }
+            // fold the partials of spans fb..lb: span f keeps its own in its staging tile, the others
+            // (which the pair entered from the left) in their parking buffers
+            float mstar[kMaxGroup], lsum[kMaxGroup];
+            float4 acc[kMaxGroup];
+#pragma unroll
+            for (int g = 0; g < kMaxGroup; ++g) { mstar[g] = -INFINITY; lsum[g] = 0.f; acc[g] = make_float4(0.f, 0.f, 0.f, 0.f); }
+            auto rows_of = [&](int sp, int &pitch) -> const float * {
+                const int w = sp - b0;
+                if (sp == f) { pitch = Lay::kStagePitch; return (const float *)(smem + Lay::kStagingOff + w * Lay::kStagingBytes); }
+                pitch = D;
+                return (const float *)(smem + Lay::kParkOff + w * Lay::kParkBytes);
+            };
+            for (int sp = fb; sp <= lb; ++sp) {
+                int pitch;
+                const float *rows = rows_of(sp, pitch);
+                const float *ml = rows + kMaxGroup * pitch;
+#pragma unroll
+                for (int g = 0; g < kMaxGroup; ++g) mstar[g] = fmaxf(mstar[g], ml[g]);
+            }
+            for (int sp = fb; sp <= lb; ++sp) {
+                int pitch;
+                const float *rows = rows_of(sp, pitch);
+                const float *ml = rows + kMaxGroup * pitch;
+#pragma unroll
+                for (int g = 0; g < kMaxGroup; ++g) {
+                    // a column that has seen no token anywhere (multi-token step) keeps -inf: factors 0
+                    const float fct = fast_exp2(ml[g] - (mstar[g] == -INFINITY ? 0.f : mstar[g]));
+                    lsum[g] += fct * ml[kMaxGroup + g];
+                    if (g < ncols && lane * 4 < D) {
+                        const float4 a = *(const float4 *)(rows + g * pitch + lane * 4);
+                        acc[g].x += fct * a.x; acc[g].y += fct * a.y; acc[g].z += fct * a.z; acc[g].w += fct * a.w;
+                    }
+                }
+            }
+            const int c_first = f / W, c_last = l / W;
+            if (c_first == c_last) {              // the pair lies inside this CTA: done
+                store_merged<D>(acc, mstar, lsum, nullptr, nullptr, pend_out[k], ncols, G, qi_stride, lane);
+                continue;
+            }
+            // partial 0 of a pair (the CTA it begins in) lives in that CTA's odd slot, the others in
+            // the even slot of their CTA
+            const int slot = (int)blockIdx.x == c_first ? 2 * (int)blockIdx.x + 1 : 2 * (int)blockIdx.x;
+            store_merged<D>(acc, mstar, lsum, p.part_acc + (size_t)slot * kMaxGroup * D, p.part_ml + slot * 2 * kMaxGroup,
+                            nullptr, ncols, G, qi_stride, lane);
+            pend_first[k] = c_first; pend_last[k] = c_last; pend_slot[k] = 2 * c_first + 1;
+        }
+    }
+
+    // ---- grid stage, in units of CTAs: whichever CTA arrives last for a (request, kv head) merges
+    // the CTAs' partials (wait-free).
     if (pend_first[0] >= 0 || pend_first[1] >= 0) {
         int n_part[2], sub[2], grp[2], grp_cnt[2], n_grp[2];
 #pragma unroll
@@ -1249,7 +1324,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             sub[k] = 0; grp[k] = 0; grp_cnt[k] = n_part[k]; n_grp[k] = 1;
             if (n_part[k] > kTreeFrom) {
                 sub[k] = merge_group_size(n_part[k]);
-                grp[k] = (span - pend_first[k]) / sub[k];
+                grp[k] = ((int)blockIdx.x - pend_first[k]) / sub[k];
                 n_grp[k] = (n_part[k] + sub[k] - 1) / sub[k];
                 grp_cnt[k] = min(sub[k], n_part[k] - grp[k] * sub[k]);
             }

@@ -1308,8 +1308,50 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             // partial 0 of a pair (the CTA it begins in) lives in that CTA's odd slot, the others in
             // the even slot of their CTA
             const int slot = (int)blockIdx.x == c_first ? 2 * (int)blockIdx.x + 1 : 2 * (int)blockIdx.x;
+            // publish this CTA's partial; the stores drain while the counter is asked
             store_merged<D>(acc, mstar, lsum, p.part_acc + (size_t)slot * kMaxGroup * D, p.part_ml + slot * 2 * kMaxGroup,
                             nullptr, ncols, G, qi_stride, lane);
+            if (c_last == c_first + 1) {
+                // Two CTAs share the pair.  If the other one has arrived already (counter at 1), its
+                // partial is published and this warp is the last: it merges straight from its
+                // registers -- one round trip for the counter, one for the other partial.  If not,
+                // it counts itself in; should the other one have arrived in between, it is the last
+                // after all and does the same.
+                int seen = 0;
+                if (lane == 0) seen = atomicCAS(p.arrivals + c_first, 1, 0);
+                seen = __shfl_sync(0xffffffffu, seen, 0);
+                if (seen != 1) {
+                    __threadfence();              // the partial's stores left before the counter was asked
+                    if (lane == 0) seen = atomicAdd(p.arrivals + c_first, 1);
+                    seen = __shfl_sync(0xffffffffu, seen, 0);
+                    if (seen != 1) continue;      // first to arrive: the other CTA merges
+                    if (lane == 0) p.arrivals[c_first] = 0;
+                }
+                __threadfence();
+                const int other = (int)blockIdx.x == c_first ? 2 * c_last : 2 * c_first + 1;
+                const float *oml = p.part_ml + other * 2 * kMaxGroup;
+                const float *oacc = p.part_acc + (size_t)other * kMaxGroup * D + lane * 4;
+                const float4 m_lo = ld_cg_f32x4(oml), m_hi = ld_cg_f32x4(oml + 4);
+                const float4 l_lo = ld_cg_f32x4(oml + 8), l_hi = ld_cg_f32x4(oml + 12);
+                float4 oa[kMaxGroup];
+#pragma unroll
+                for (int g = 0; g < kMaxGroup; ++g)
+                    oa[g] = (g < ncols && lane * 4 < D) ? ld_cg_f32x4(oacc + g * D) : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float om[kMaxGroup] = {m_lo.x, m_lo.y, m_lo.z, m_lo.w, m_hi.x, m_hi.y, m_hi.z, m_hi.w};
+                const float ol[kMaxGroup] = {l_lo.x, l_lo.y, l_lo.z, l_lo.w, l_hi.x, l_hi.y, l_hi.z, l_hi.w};
+#pragma unroll
+                for (int g = 0; g < kMaxGroup; ++g) {
+                    const float mx = fmaxf(mstar[g], om[g]);
+                    const float ref = mx == -INFINITY ? 0.f : mx;
+                    const float fa = fast_exp2(mstar[g] - ref), fo = fast_exp2(om[g] - ref);
+                    mstar[g] = mx;
+                    lsum[g] = fa * lsum[g] + fo * ol[g];
+                    acc[g].x = fa * acc[g].x + fo * oa[g].x; acc[g].y = fa * acc[g].y + fo * oa[g].y;
+                    acc[g].z = fa * acc[g].z + fo * oa[g].z; acc[g].w = fa * acc[g].w + fo * oa[g].w;
+                }
+                store_merged<D>(acc, mstar, lsum, nullptr, nullptr, pend_out[k], ncols, G, qi_stride, lane);
+                continue;
+            }
             pend_first[k] = c_first; pend_last[k] = c_last; pend_slot[k] = 2 * c_first + 1;
         }
     }

@@ -21,7 +21,7 @@ constexpr int kMaxGroup = 8;         // query heads per KV head handled by one M
 constexpr int kMaxSpans = 2048;      // upper bound on the partition width (one span per warp)
 constexpr int kMaxBatch = 8192;
 constexpr int kBulkMergeFrom = 4;    // merges of more partials than this go through shared memory
-constexpr int kTreeFrom = 12;        // pairs cut into more partials than this are merged in two levels
+constexpr int kTreeFrom = 24;        // pairs cut into more partials than this are merged in two levels
 
 constexpr uint32_t kStatusBadLength = 1u;
 constexpr uint32_t kStatusBadPage = 2u;
@@ -1251,7 +1251,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     // CTA the result is final; otherwise it is the CTA's one partial of the pair for the grid stage.
     {
         const int b0 = blockIdx.x * W;
-#pragma unroll
+#pragma unroll 1                                      // executed once per warp: keep the code small, it runs from a cold instruction cache
         for (int k = 0; k < 2; ++k) {
             if (pend_first[k] < 0) continue;
             const int f = pend_first[k], l = pend_last[k];

@@ -306,6 +306,24 @@ def test_attention_kernel_derives_the_same_partition_as_the_plan():
     assert ds.pool.check_status() == 0
 
 
+# --------------------------------------------------------------------------- merge stages
+
+@pytest.mark.parametrize("Hq,Hkv", [(4, 1), (8, 1), (8, 2)])
+def test_every_merge_stage_matches_oracle(Hq, Hkv):
+    """One long context cut into C spans exercises each way partials are merged: inside one CTA
+    through shared memory (C <= 4 spans), two CTAs with the later one merging from its registers
+    (5..8), a flat merge of up to 24 CTA partials, and the two-level merge beyond that -- with a
+    short request behind it so that the last span also holds a whole (request, kv head)."""
+    h = custom_inputs([9000, 70], Hq, Hkv, 128, seed=500 + Hq + Hkv)
+    ref_pool, ref_out = oracle_step(h)
+    for fused in (False, True):
+        for C in (1, 2, 3, 4, 5, 6, 8, 9, 12, 40, 96, 97, 130, 400):
+            ds = run_step(h, partition=C, fused=fused)
+            assert np.array_equal(dev_to_bits(ds.pool.pool), ref_pool)
+            assert_close(dev_to_bits(ds.out[0]), ref_out, "merge stages C=%d fused=%s" % (C, fused))
+            ds.pool.close()
+
+
 # --------------------------------------------------------------------------- configs 2, 5
 
 def device_workload(name, batch=None, num_layers=None):

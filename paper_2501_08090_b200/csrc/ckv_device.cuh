@@ -334,11 +334,20 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     }
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar)
+// L2 policy for data that is read once: such lines are the first to be evicted, so the stream of KV
+// tiles does not push tables, queries and partial results out of the cache.
+__device__ __forceinline__ uint64_t l2_evict_first_policy()
+{
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar, uint64_t policy)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
 }
 
 // Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
@@ -904,6 +913,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     unsigned long long t_issue = 0, t_masked = 0;
 #endif
     bool inputs_ready = true;                    // q, k_new and v_new may be read (the dependency wait is behind us)
+    const uint64_t kv_policy = l2_evict_first_policy();
     auto issue_next = [&]() {
 #ifdef CKV_TRACE_WAITS
         const unsigned long long i0 = global_timer_ns();
@@ -931,7 +941,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             }
             const int y = ((p.layer_page_base + src_page) * p.num_kv_heads + ic.h) * 32;
             tma_load_2d(ring + slot * Lay::kStageBytes + pg * Lay::kPageBytes + hf * Lay::kHalfBytes,
-                        &tmap, hf * 64, y, bars + slot * 8);
+                        &tmap, hf * 64, y, bars + slot * 8, kv_policy);
         }
         if (p.k_new != nullptr && ic.tile == ic.tiles - 1 && an_r < 0 && inputs_ready) {
             // last tile of this (request, kv head): fetch the rows to append and remember their page

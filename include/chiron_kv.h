@@ -194,10 +194,13 @@ int32_t ckv_set_overlap(ckv_pool *pool, int32_t enable);
 int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits);
 
 /*
- * One whole iteration for one layer with HOST buffers (pinned memory recommended): copies the
- * tables, lengths, q, k_new and v_new to the device, runs decode_step, copies
- * the output back and synchronises `stream`.  h_out: bf16 [batch][num_q_heads][head_dim].
- * Errors: as kv_append / decode_attention.
+ * One whole iteration for one layer with HOST buffers: brings the tables, lengths, q, k_new and
+ * v_new to the device, runs decode_step, delivers the output to h_out and synchronises `stream`.
+ * If the device can address all six buffers (pinned or registered host memory, h_out 16-byte
+ * aligned) nothing is copied by DMA: one kernel gathers the five inputs into the workspace and
+ * the attention kernel writes its output rows straight into h_out (two launches); otherwise five
+ * host-to-device copies, decode_step and one device-to-host copy are issued.
+ * h_out: bf16 [batch][num_q_heads][head_dim].  Errors: as kv_append / decode_attention.
  */
 int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch,
                          const int32_t *h_block_tables, const int32_t *h_seq_lens,

@@ -517,6 +517,18 @@ int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits)
     return CKV_OK;
 }
 
+// Device-visible address of a host buffer if the device can address it (pinned or registered
+// memory), else NULL.
+static void *mapped_or_null(const void *h)
+{
+    void *d = nullptr;
+    if (cudaHostGetDevicePointer(&d, const_cast<void *>(h), 0) != cudaSuccess) {
+        cudaGetLastError();                      // not an error of the caller's: the copy path is taken
+        return nullptr;
+    }
+    return d;
+}
+
 int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *h_block_tables,
                          const int32_t *h_seq_lens, const void *h_q, const void *h_k_new,
                          const void *h_v_new, void *h_out, void *stream)
@@ -531,13 +543,48 @@ int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch, const int
     int32_t *d_sl = pool->wsp<int32_t>(pool->ws.st_lens);
     void *d_q = pool->d_ws + pool->ws.st_q, *d_k = pool->d_ws + pool->ws.st_k;
     void *d_v = pool->d_ws + pool->ws.st_v, *d_o = pool->d_ws + pool->ws.st_out;
-    CKV_CUDA(cudaMemcpyAsync(d_bt, h_block_tables, sizeof(int32_t) * (size_t)batch * c.max_pages_per_req, cudaMemcpyHostToDevice, s));
-    CKV_CUDA(cudaMemcpyAsync(d_sl, h_seq_lens, sizeof(int32_t) * (size_t)batch, cudaMemcpyHostToDevice, s));
-    CKV_CUDA(cudaMemcpyAsync(d_q, h_q, (size_t)batch * c.num_q_heads * d2, cudaMemcpyHostToDevice, s));
-    CKV_CUDA(cudaMemcpyAsync(d_k, h_k_new, (size_t)batch * c.num_kv_heads * d2, cudaMemcpyHostToDevice, s));
-    CKV_CUDA(cudaMemcpyAsync(d_v, h_v_new, (size_t)batch * c.num_kv_heads * d2, cudaMemcpyHostToDevice, s));
+    const size_t n_bt = sizeof(int32_t) * (size_t)batch * c.max_pages_per_req, n_sl = sizeof(int32_t) * (size_t)batch;
+    const size_t n_q = (size_t)batch * c.num_q_heads * d2, n_kv = (size_t)batch * c.num_kv_heads * d2;
+
+    // Pinned buffers the device can address: one gather kernel brings all five inputs over, and
+    // the attention kernel writes its output rows straight into the host buffer -- two launches
+    // instead of six copies and one.  The tables and lengths come from the kernel just before, so
+    // this launch takes plain stream order.
+    const void *m_bt = mapped_or_null(h_block_tables), *m_sl = mapped_or_null(h_seq_lens), *m_q = mapped_or_null(h_q);
+    const void *m_k = mapped_or_null(h_k_new), *m_v = mapped_or_null(h_v_new);
+    void *m_o = mapped_or_null(h_out);
+    if (m_bt && m_sl && m_q && m_k && m_v && m_o && aligned16(m_o)) {
+        ckv::GatherParams gp{};
+        const void *src[5] = {m_bt, m_sl, m_q, m_k, m_v};
+        void *dst[5] = {d_bt, d_sl, d_q, d_k, d_v};
+        const size_t bytes[5] = {n_bt, n_sl, n_q, n_kv, n_kv};
+        size_t total = 0;
+        for (int a = 0; a < 5; ++a) {
+            gp.src[a] = static_cast<const uint8_t *>(src[a]);
+            gp.dst[a] = static_cast<uint8_t *>(dst[a]);
+            gp.bytes[a] = bytes[a];
+            total += bytes[a];
+        }
+        const int blocks = (int)std::min<size_t>((total / 16 + 255) / 256 + 1, (size_t)pool->num_sms * 8);
+        ckv::host_gather_kernel<<<blocks, 256, 0, s>>>(gp);
+        CKV_CUDA(cudaGetLastError());
+        pool->launches += 1;
+        const bool overlap = pool->overlap;
+        pool->overlap = false;
+        const int32_t rc = decode_step(pool, layer, batch, d_bt, d_sl, d_q, d_k, d_v, m_o, stream);
+        pool->overlap = overlap;
+        if (rc) return rc;
+        CKV_CUDA(cudaStreamSynchronize(s));
+        return CKV_OK;
+    }
+
+    CKV_CUDA(cudaMemcpyAsync(d_bt, h_block_tables, n_bt, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(d_sl, h_seq_lens, n_sl, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(d_q, h_q, n_q, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(d_k, h_k_new, n_kv, cudaMemcpyHostToDevice, s));
+    CKV_CUDA(cudaMemcpyAsync(d_v, h_v_new, n_kv, cudaMemcpyHostToDevice, s));
     if (int32_t rc = decode_step(pool, layer, batch, d_bt, d_sl, d_q, d_k, d_v, d_o, stream)) return rc;
-    CKV_CUDA(cudaMemcpyAsync(h_out, d_o, (size_t)batch * c.num_q_heads * d2, cudaMemcpyDeviceToHost, s));
+    CKV_CUDA(cudaMemcpyAsync(h_out, d_o, n_q, cudaMemcpyDeviceToHost, s));
     CKV_CUDA(cudaStreamSynchronize(s));
     return CKV_OK;
 }

@@ -151,6 +151,34 @@ __global__ void kv_swap_kernel(const SwapParams p)
 }
 
 // ------------------------------------------------------------------------------------------
+// Gather of one step's inputs from pinned host memory that the device addresses directly: up to
+// five arrays (tables, lengths, q, new keys, new values) move to their device staging areas in one
+// launch instead of one DMA copy each.  Sizes are multiples of 4 bytes.
+// ------------------------------------------------------------------------------------------
+struct GatherParams {
+    const uint8_t *src[5];
+    uint8_t *dst[5];
+    unsigned long long bytes[5];
+};
+
+__global__ void host_gather_kernel(const GatherParams p)
+{
+    const size_t tid = blockIdx.x * (size_t)blockDim.x + threadIdx.x, nthr = (size_t)gridDim.x * blockDim.x;
+#pragma unroll
+    for (int a = 0; a < 5; ++a) {
+        const uint8_t *src = p.src[a];
+        uint8_t *dst = p.dst[a];
+        const size_t bytes = p.bytes[a];
+        const bool vec = ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15u) == 0;
+        const size_t nvec = vec ? bytes / 16 : 0;
+        for (size_t i = tid; i < nvec; i += nthr)
+            reinterpret_cast<uint4 *>(dst)[i] = reinterpret_cast<const uint4 *>(src)[i];
+        for (size_t i = nvec * 4 + tid; i < bytes / 4; i += nthr)
+            reinterpret_cast<uint32_t *>(dst)[i] = reinterpret_cast<const uint32_t *>(src)[i];
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // Cache flush helper of the latency sweep: read `vecs` 16-byte pieces once.  Run after a buffer
 // larger than the L2 has been overwritten, it replaces the dirty lines that the overwrite left
 // in the cache by clean ones, so the step timed next does not pay for their write-back.

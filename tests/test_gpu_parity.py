@@ -405,19 +405,26 @@ def test_skewed_long_context_full_parity():
 
 # --------------------------------------------------------------------------- host-buffer entry and sweep
 
-def test_decode_step_host_matches_oracle():
+@pytest.mark.parametrize("pinned", [True, False])
+def test_decode_step_host_matches_oracle(pinned):
+    """Pinned buffers take the zero-copy route (gather kernel in, output rows written straight to
+    the host buffer), pageable ones the copy route; both must give the oracle's step."""
     h = wl.host_inputs(wl.workload("tiny"))
     ref_pool, ref_out = oracle_step(h)
     ds = make_device_step(h)
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    host = lambda a: torch.from_numpy(np.ascontiguousarray(a).copy())
+    pin = (lambda a: host(a).pin_memory()) if pinned else host
     q = pin(h.q[0].view(np.int16)).view(torch.bfloat16)
     k = pin(h.k_new[0].view(np.int16)).view(torch.bfloat16)
     v = pin(h.v_new[0].view(np.int16)).view(torch.bfloat16)
-    out = torch.zeros_like(q).pin_memory()
+    out = torch.zeros_like(q)
+    out = out.pin_memory() if pinned else out
+    n0 = ds.pool.launch_count()
     ds.pool.decode_step_host(0, pin(h.block_tables), pin(h.seq_lens), q, k, v, out)
+    assert ds.pool.launch_count() - n0 == (2 if pinned else 1)
     assert ds.pool.check_status() == 0
     assert np.array_equal(dev_to_bits(ds.pool.pool), ref_pool)
-    assert_close(dev_to_bits(out), ref_out, "decode_step_host")
+    assert_close(dev_to_bits(out), ref_out, "decode_step_host pinned=%s" % pinned)
 
 
 def test_step_latency_sweep_runs_nested_prefixes_and_counts_launches():

@@ -139,10 +139,13 @@ int32_t decode_step(ckv_pool *pool, int32_t layer, int32_t batch,
  * the q_len tokens are appended; requests with seq_lens[r] < q_len are unusable (status bit, rows
  * zero-filled).
  *   kv_append_multi         d_k_new, d_v_new: bf16 [batch][q_len][num_kv_heads][head_dim]; 1 <= q_len <= 8
- *   decode_attention_multi  d_q, d_out: bf16 [batch][q_len][num_q_heads][head_dim]; the new tokens'
- *                           queries share the 8 columns of one tensor-core pass with the heads of
- *                           the group, so the KV stream is read once for all of them; this needs
- *                           q_len * (num_q_heads / num_kv_heads) <= 8, otherwise CKV_EINVAL.
+ *   decode_attention_multi  d_q, d_out: bf16 [batch][q_len][num_q_heads][head_dim]; 1 <= q_len <= 8.
+ *                           The new tokens' queries share the 8 columns of one tensor-core pass
+ *                           with the heads of the group, so while
+ *                           q_len * (num_q_heads / num_kv_heads) <= 8 the KV stream is read once
+ *                           for all of them.  Beyond that the step takes
+ *                           ceil(q_len / (8 / group)) launches, each reading the KV stream again for
+ *                           its own block of new tokens.
  * Call kv_append_multi first: attention reads the new tokens' keys and values from the pool.
  * Errors: CKV_EINVAL, CKV_ECUDA.
  */

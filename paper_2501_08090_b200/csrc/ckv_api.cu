@@ -395,9 +395,7 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
                                 const void *d_k_new, const void *d_v_new, void *d_out, void *stream)
 {
     if (int32_t rc = check_call(pool, layer, batch, fn)) return rc;
-    if (q_len < 1 || q_len * (pool->cfg.num_q_heads / pool->cfg.num_kv_heads) > ckv::kMaxGroup)
-        return fail(CKV_EINVAL, "%s: q_len %d x group %d exceeds the %d columns one pass holds", fn, q_len,
-                    pool->cfg.num_q_heads / pool->cfg.num_kv_heads, ckv::kMaxGroup);
+    if (q_len < 1 || q_len > ckv::kMaxGroup) return fail(CKV_EINVAL, "%s: q_len %d outside [1, %d]", fn, q_len, ckv::kMaxGroup);
     if (q_len > 1 && d_k_new) return fail(CKV_EINVAL, "%s: the fused append is for single-token steps", fn);
     if (!d_block_tables || !d_seq_lens || !d_q || !d_out) return fail(CKV_EINVAL, "%s: NULL argument", fn);
     if (!aligned16(d_q) || !aligned16(d_out)) return fail(CKV_EINVAL, "%s: q/out not 16-byte aligned", fn);
@@ -430,6 +428,8 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
     ap.layer_page_base = layer * c.num_pages;
     ap.num_spans = pool->num_spans;
     ap.q_len = q_len;
+    ap.q_base = 0;
+    ap.q_pass = q_len;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
 
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -446,16 +446,23 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
         pool->ev_used += 1;
         CKV_CUDA(cudaEventRecord(ev0, s));
     }
-    int32_t rc;
-    if (c.head_dim == 128)
-        rc = q_len > 1 ? launch_attention<128, kWarps128, kStages128, true>(pool, ap, s)
-                       : launch_attention<128, kWarps128, kStages128, false>(pool, ap, s);
-    else
-        rc = q_len > 1 ? launch_attention<64, kWarps64, kStages64, true>(pool, ap, s)
-                       : launch_attention<64, kWarps64, kStages64, false>(pool, ap, s);
-    if (rc) return rc;
+    // One launch holds 8 (new token, head) columns: 8 / group new tokens.  More new tokens take
+    // more launches, each streaming the KV again for its own block of new tokens.
+    const int per_pass = ckv::kMaxGroup / ap.group;
+    for (int base = 0; base < q_len; base += per_pass) {
+        ap.q_base = base;
+        ap.q_pass = std::min(per_pass, q_len - base);
+        int32_t rc;
+        if (c.head_dim == 128)
+            rc = q_len > 1 ? launch_attention<128, kWarps128, kStages128, true>(pool, ap, s)
+                           : launch_attention<128, kWarps128, kStages128, false>(pool, ap, s);
+        else
+            rc = q_len > 1 ? launch_attention<64, kWarps64, kStages64, true>(pool, ap, s)
+                           : launch_attention<64, kWarps64, kStages64, false>(pool, ap, s);
+        if (rc) return rc;
+        pool->launches += 1;
+    }
     if (ev1) CKV_CUDA(cudaEventRecord(ev1, s));
-    pool->launches += 1;
     return CKV_OK;
 }
 
@@ -771,6 +778,8 @@ int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int3
     ap.layer_page_base = layer * cfg->num_pages;
     ap.num_spans = num_spans;
     ap.q_len = 1;
+    ap.q_base = 0;
+    ap.q_pass = 1;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)cfg->head_dim));
 
     int32_t rc;

@@ -518,14 +518,17 @@ struct AttnParams {
     int32_t batch, max_pages_per_req, num_pages, num_kv_heads, num_q_heads, group;
     int32_t layer_page_base;        // layer * num_pages
     int32_t num_spans;
-    int32_t q_len;                  // new tokens per request in this step (1 for plain decode); q_len*group <= 8
+    int32_t q_len;                  // new tokens per request in this step (1 for plain decode)
+    int32_t q_base, q_pass;         // this launch computes new tokens q_base .. q_base + q_pass - 1; q_pass*group <= 8
     float scale_log2;               // log2(e) / sqrt(d)
 };
 
 // Columns.  The 8 columns of the MMA hold (new token, head of the group) pairs: column c is new
-// token c / G and head c % G, ncols = q_len * G <= 8 of them are live.  With one new token per
-// request (the usual decode step) a column is simply a head.  Output rows of a (request, kv head)
-// start at out_rows; column c's row is out_rows + (c / G) * qi_stride + (c % G) * D.
+// token q_base + c / G and head c % G, ncols = q_pass * G <= 8 of them are live.  A step with more
+// new tokens than fit is run as several launches, each over the whole KV stream with its own
+// q_base.  With one new token per request (the usual decode step) a column is simply a head.
+// Output rows of a (request, kv head) start at out_rows (new token q_base); column c's row is
+// out_rows + (c / G) * qi_stride + (c % G) * D.
 //
 // Merge the partials of one (request, kv head) that spans s_first..s_last hold, and write its bf16
 // output rows.  Run by one whole warp (the last one to arrive for that pair).  Loads are issued in
@@ -890,7 +893,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     const long long v_end = st.end;
     const int q_span = st.q;
     const int G = p.group;
-    const int ncols = G * p.q_len;               // live MMA columns: column c = new token c / G, head c % G
+    const int ncols = G * p.q_pass;              // live MMA columns: column c = new token q_base + c / G, head c % G
     const int qi_stride = p.num_q_heads * D;     // elements between a request's consecutive new tokens in q / out
 
     // ---- issue side: block-table entries travel in registers, 32 pages (16 tiles) per chunk
@@ -917,7 +920,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     int qn_r = -1, qn_h = -1;
     const int c_row = lane >> 2;                 // the column this lane loads Q for
     auto load_q = [&](uint32_t (&dst)[Lay::kKSteps][2], int r, int h) {
-        const uint32_t *qrow = (const uint32_t *)(p.q + ((size_t)r * p.q_len + c_row / G) * qi_stride +
+        const uint32_t *qrow = (const uint32_t *)(p.q + ((size_t)r * p.q_len + p.q_base + c_row / G) * qi_stride +
                                                   (size_t)(h * G + c_row % G) * D);
 #pragma unroll
         for (int ks = 0; ks < Lay::kKSteps; ++ks) {
@@ -1084,12 +1087,12 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             if (done == 0 && lane == 0) p.trace[span * 8 + 1] = global_timer_ns();
 
             const int ntok = min(kTileTokens, piece_L - ti * kTileTokens);      // tokens of the context in this tile
-            // Causality among the step's new tokens: column c (new token c / G) sees the context up to
-            // and including its own position, i.e. vis_all + c / G tokens; every column sees vis_all.
+            // Causality among the step's new tokens: column c (new token t = q_base + c / G) sees the
+            // context up to and including its own position, i.e. vis_all + t tokens; every column sees vis_all.
             const int vis_all = kMulti ? piece_L - p.q_len + 1 : piece_L;
             const bool full_tile = (ti + 1) * kTileTokens <= vis_all;
-            const int lim0 = kMulti ? min(ntok, vis_all + qi0 - ti * kTileTokens) : ntok;   // visible tokens of this tile,
-            const int lim1 = kMulti ? min(ntok, vis_all + qi1 - ti * kTileTokens) : ntok;   // for this lane's two columns
+            const int lim0 = kMulti ? min(ntok, vis_all + p.q_base + qi0 - ti * kTileTokens) : ntok;   // visible tokens of this tile,
+            const int lim1 = kMulti ? min(ntok, vis_all + p.q_base + qi1 - ti * kTileTokens) : ntok;   // for this lane's two columns
             const int np = (ntok + kPageSize - 1) / kPageSize;
             const uint32_t sb = ring + slot * Lay::kStageBytes;
 
@@ -1232,7 +1235,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             staging[(g0 + 1) * Lay::kStagePitch + d + 8] = o[dt][3];
         }
         __syncwarp();
-        uint16_t *out_rows = p.out + (size_t)piece_r * p.q_len * qi_stride + (size_t)piece_h * G * D;
+        uint16_t *out_rows = p.out + ((size_t)piece_r * p.q_len + p.q_base) * qi_stride + (size_t)piece_h * G * D;
         if (complete) {
 #pragma unroll
             for (int g = 0; g < kMaxGroup; ++g) {

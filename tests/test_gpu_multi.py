@@ -50,7 +50,9 @@ EDGE_LENS = [8, 9, 15, 16, 17, 31, 32, 33, 34, 35, 36, 47, 48, 49, 63, 64, 65, 6
 
 
 @pytest.mark.parametrize("q_len,Hq,Hkv,d", [(2, 8, 2, 128), (2, 32, 8, 128), (4, 4, 2, 128), (4, 2, 1, 64),
-                                            (8, 2, 2, 128), (8, 1, 1, 64), (3, 4, 2, 64), (1, 8, 1, 128)])
+                                            (8, 2, 2, 128), (8, 1, 1, 64), (3, 4, 2, 64), (1, 8, 1, 128),
+                                            # more (new token, head) pairs than one launch holds: 2, 3, 4 and 8 passes
+                                            (3, 32, 8, 128), (5, 8, 2, 128), (4, 8, 1, 128), (8, 16, 2, 64)])
 def test_multi_token_step_matches_oracle(q_len, Hq, Hkv, d):
     lens = [L for L in EDGE_LENS if L >= q_len]
     run_case(q_len, Hq, Hkv, d, lens, seed=q_len * 100 + Hq, partitions=(None, 1, 11, 2048))
@@ -76,12 +78,16 @@ def test_multi_token_limits_are_checked_on_the_host():
     from paper_2501_08090_b200 import binding as b
     cfg = b.make_config(1, 32, 8, 128, 16, 4, 2)
     kp = b.KvPool(cfg)
-    z = torch.zeros(2, 3, 32, 128, dtype=torch.bfloat16, device="cuda")
+    z = torch.zeros(2, 9, 32, 128, dtype=torch.bfloat16, device="cuda")
     bt = torch.zeros(2, 4, dtype=torch.int32, device="cuda")
     sl = torch.full((2,), 10, dtype=torch.int32, device="cuda")
-    with pytest.raises(b.CkvError) as e:
-        kp.decode_attention_multi(0, 3, bt, sl, z, z.clone())   # 3 new tokens x group 4 > 8 columns
-    assert e.value.code == b.CKV_EINVAL and "columns" in str(e.value)
+    for bad in (0, 9):
+        with pytest.raises(b.CkvError) as e:
+            kp.decode_attention_multi(0, bad, bt, sl, z, z.clone())
+        assert e.value.code == b.CKV_EINVAL and "q_len" in str(e.value)
+    n0 = kp.launch_count()
+    kp.decode_attention_multi(0, 3, bt, sl, z[:, :3].contiguous(), z[:, :3].clone())   # 3 new tokens x group 4: two passes
+    assert kp.launch_count() - n0 == 2
     kp.close()
 
 

@@ -398,6 +398,10 @@ def run_ours(args) -> None:
             line["global_autoscaler"] = run_global_autoscaler(line["local_autoscaler"])
             line["kv_swap"] = run_swap(dev)
             line["multi_token_step"] = run_multi_token(dw)
+            dw.kp.close()
+            del dw
+            torch.cuda.empty_cache()
+            line["other_workloads"] = run_other_workloads(dev)
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(HEADLINE)
     if rank == 0:
@@ -459,10 +463,10 @@ def run_swap(dev) -> dict:
 
 def run_multi_token(dw) -> dict:
     """kv_append_multi + decode_attention_multi on the headline batch: q_len new tokens per request
-    share one pass over the KV stream (q_len x group <= 8 columns)."""
+    share one pass over the KV stream while q_len x group <= 8 columns; q_len 4 takes two passes."""
     import torch
     w, rows = dw.w, []
-    for q_len in range(1, 8 // w.group + 1):
+    for q_len in (1, 2, 4):
         q = wl.device_normal_bf16((dw.B, q_len, w.num_q_heads, w.head_dim), w.seed, 20 + q_len, dw.device)
         k = wl.device_normal_bf16((dw.B, q_len, w.num_kv_heads, w.head_dim), w.seed, 30 + q_len, dw.device)
         out = torch.zeros_like(q)
@@ -480,10 +484,44 @@ def run_multi_token(dw) -> dict:
             step()
         e1.record(); torch.cuda.synchronize()
         us = e0.elapsed_time(e1) * 1e3 / n
-        rows.append({"q_len": q_len, "us_per_step": round(us, 2), "kv_tbs": round(dw.bytes["kv"] / us / 1e6, 3),
+        passes = -(-q_len * w.group // 8)
+        rows.append({"q_len": q_len, "passes": passes, "us_per_step": round(us, 2),
+                     "kv_tbs": round(passes * dw.bytes["kv"] / us / 1e6, 3),
                      "new_tokens_per_s": round(dw.B * q_len / us * 1e6)})
     dw.kp.check_status()
-    return {"workload": dw.w.name, "launches_per_step": 2, "points": rows}
+    return {"workload": dw.w.name, "launches_per_step": "1 append + passes", "points": rows}
+
+
+def run_other_workloads(dev) -> list:
+    """The other full-size workloads, back to back like the headline: the skewed long-context batch
+    and the 70B-shaped iteration with all 80 layers resident (about 80 GB of KV)."""
+    import torch
+    rows = []
+    for name, steps in (("skewed_long", 300), ("llama70b_full", 5)):
+        try:
+            dw = DeviceWorkload(name, dev)
+        except torch.cuda.OutOfMemoryError:
+            rows.append({"workload": name, "skipped": "not enough free device memory"})
+            continue
+        dw.run_steps(2)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        dw.run_steps(steps)
+        e1.record()
+        torch.cuda.synchronize()
+        dw.kp.check_status()
+        us = e0.elapsed_time(e1) * 1e3 / steps
+        tbs = dw.bytes["total"] / us / 1e6
+        rows.append({"workload": name, "batch": dw.B, "layers": dw.w.num_layers, "steps": steps,
+                     "us_per_step": round(us, 1), "us_per_layer": round(us / dw.w.num_layers, 2),
+                     "tokens_per_s": round(dw.B / us * 1e6), "tbs": round(tbs, 3),
+                     "frac_of_8TBs": round(tbs / NORMALISED_TO_TBS, 4),
+                     "kv_bytes_per_step": int(dw.bytes["kv"])})
+        dw.kp.close()
+        del dw
+        torch.cuda.empty_cache()
+    return rows
 
 
 def run_autoscaler(sweep: dict) -> dict:

@@ -185,10 +185,12 @@ int32_t ckv_get_partition(const ckv_pool *pool);
  * they must not be produced by the kernel that immediately precedes decode_attention in the
  * stream (tables copied by a memcpy, or written by any earlier kernel, are fine -- the usual case,
  * since a serving engine uploads them once per iteration).  decode_step, being the only writer of
- * its layer's pool, also starts its first KV tile loads before that wait: with overlap on, the
- * kernel that immediately precedes decode_step must not write pool pages that this step reads,
- * unless it is a decode_step itself (whose appended rows this step replaces in its staged tiles
- * anyway).  Turning overlap off restores plain stream order.  Errors: CKV_EINVAL. */
+ * its layer's pool, also starts its first KV tile loads before that wait: with overlap on, a
+ * kernel of the CALLER's that immediately precedes decode_step must not write pool pages that
+ * this step reads.  The library's own writers are taken care of: after kv_append,
+ * kv_append_multi or kv_swap_in on this handle the next decode_step waits before its loads, and
+ * a preceding decode_step's appended rows are replaced in this step's staged tiles anyway.
+ * Turning overlap off restores plain stream order.  Errors: CKV_EINVAL. */
 int32_t ckv_set_overlap(ckv_pool *pool, int32_t enable);
 
 /* Synchronise `stream`, read and clear the device status word.  Returns CKV_OK, CKV_EBOUNDS

@@ -125,6 +125,7 @@ struct ckv_pool {
     int64_t launches;
     bool profile;
     bool overlap;                    // launch kernels with programmatic stream serialization
+    bool pool_written;               // a kernel other than the fused step wrote the pool since the last attention launch
     std::vector<cudaEvent_t> ev;     // pairs (start, stop)
     int ev_used;
 
@@ -273,6 +274,7 @@ int32_t kv_pool_create(const ckv_config *cfg, void *d_pool, size_t pool_bytes, v
     p->launches = 0;
     p->profile = false;
     p->overlap = true;
+    p->pool_written = false;
     p->ev_used = 0;
 
     // Tensor map over the whole pool seen as rows of head_dim bf16; one box = 32 rows (the 16 key
@@ -373,6 +375,7 @@ static int32_t append_launch(ckv_pool *pool, const char *fn, int32_t layer, int3
     lc.numAttrs = 1;
     CKV_CUDA(cudaLaunchKernelEx(&lc, ckv::kv_append_kernel, ap));
     pool->launches += 1;
+    pool->pool_written = true;
     return CKV_OK;
 }
 
@@ -430,6 +433,10 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
     ap.q_len = q_len;
     ap.q_base = 0;
     ap.q_pass = q_len;
+    // A fused step may start loading tiles under its predecessor's tail -- unless that predecessor
+    // may be a kernel of this library that writes the pool (an append or a swap-in).
+    ap.early_loads = pool->pool_written ? 0 : 1;
+    pool->pool_written = false;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
 
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -780,6 +787,7 @@ int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int3
     ap.q_len = 1;
     ap.q_base = 0;
     ap.q_pass = 1;
+    ap.early_loads = 0;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)cfg->head_dim));
 
     int32_t rc;
@@ -828,6 +836,7 @@ static int32_t swap_launch(ckv_pool *pool, const char *fn, bool to_host, int32_t
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (to_host) ckv::kv_swap_kernel<true><<<blocks, threads, 0, s>>>(sp);
     else ckv::kv_swap_kernel<false><<<blocks, threads, 0, s>>>(sp);
+    if (!to_host) pool->pool_written = true;
     CKV_CUDA(cudaGetLastError());
     pool->launches += 1;
     return CKV_OK;

@@ -519,6 +519,7 @@ struct AttnParams {
     int32_t layer_page_base;        // layer * num_pages
     int32_t num_spans;
     int32_t q_len;                  // new tokens per request in this step (1 for plain decode)
+    int32_t early_loads;            // the first tile loads may be issued before the dependency wait (fused step only)
     int32_t q_base, q_pass;         // this launch computes new tokens q_base .. q_base + q_pass - 1; q_pass*group <= 8
     float scale_log2;               // log2(e) / sqrt(d)
 };
@@ -1006,7 +1007,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     // not depend on whether a tile's copy saw this step's new rows (they are put into the staged
     // tile before use).  Its first loads can therefore start before the preceding kernel has
     // finished -- under that kernel's tail -- as long as nothing of q, k_new or v_new is touched yet.
-    const bool early = p.k_new != nullptr;
+    const bool early = p.k_new != nullptr && p.early_loads != 0;
     if (early) {
         inputs_ready = false;
         for (int k = 0; k < NS && more_to_issue; ++k) issue_next();

@@ -1387,9 +1387,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     const float ref = mx == -INFINITY ? 0.f : mx;
                     const float fa = fast_exp2(mstar[g] - ref), fo = fast_exp2(om[g] - ref);
                     mstar[g] = mx;
-                    lsum[g] = fa * lsum[g] + fo * ol[g];
-                    acc[g].x = fa * acc[g].x + fo * oa[g].x; acc[g].y = fa * acc[g].y + fo * oa[g].y;
-                    acc[g].z = fa * acc[g].z + fo * oa[g].z; acc[g].w = fa * acc[g].w + fo * oa[g].w;
+                    // products rounded separately, then added: the result is the same bits whichever
+                    // of the two CTAs does the merge
+                    lsum[g] = __fadd_rn(__fmul_rn(fa, lsum[g]), __fmul_rn(fo, ol[g]));
+                    acc[g].x = __fadd_rn(__fmul_rn(fa, acc[g].x), __fmul_rn(fo, oa[g].x));
+                    acc[g].y = __fadd_rn(__fmul_rn(fa, acc[g].y), __fmul_rn(fo, oa[g].y));
+                    acc[g].z = __fadd_rn(__fmul_rn(fa, acc[g].z), __fmul_rn(fo, oa[g].z));
+                    acc[g].w = __fadd_rn(__fmul_rn(fa, acc[g].w), __fmul_rn(fo, oa[g].w));
                 }
                 store_merged<D>(acc, mstar, lsum, nullptr, nullptr, pend_out[k], ncols, G, qi_stride, lane);
                 continue;

@@ -476,11 +476,11 @@ __device__ __forceinline__ float4 ld_cg_f32x4(const float *p)
 // K3 + K4: paged partial attention with the log-sum-exp combine folded in.
 //
 // Every WARP is an independent worker: it owns one span of the plan, a private ring of NS stages
-// in shared memory with one mbarrier per stage, and a small staging tile.  A stage holds one tile
-// (2 pages: 32 key rows and 32 value rows of one kv head).  The warp itself issues the TMA box
-// loads of the tile NS stages ahead of the one it computes on (an "issue" cursor and a "compute"
-// cursor walk the same span), so there is no producer warp, no cross-warp merge and no CTA-wide
-// barrier anywhere; a CTA is just W such warps sharing an SM's shared memory.
+// in shared memory with one mbarrier per stage, a small staging tile and a parking buffer.  A stage
+// holds one tile (2 pages: 32 key rows and 32 value rows of one kv head).  The warp itself issues
+// the TMA box loads of the tile NS stages ahead of the one it computes on (an "issue" cursor and a
+// "compute" cursor walk the same span), so there is no producer warp and, after one barrier at the
+// kernel's start, no CTA-wide synchronisation; a CTA is W such warps sharing an SM's shared memory.
 //
 // MMA formulation (operands swapped so the tile's tokens fill the M dimension):
 //   S^T[tok 16 x g 8]  = K[tok 16 x d] . Q^T[d x g 8]          (A = K rows via ldmatrix)
@@ -495,9 +495,13 @@ __device__ __forceinline__ float4 ld_cg_f32x4(const float *p)
 // after the store landed.  No other warp reads that slot as a live token in this launch.
 //
 // A piece is the part of one (request, kv head) that falls inside the span.  When it covers the
-// whole context the warp normalises and writes the bf16 output rows itself.  Otherwise it stores
-// an fp32 partial (m, l, O) and bumps an arrival counter; whichever warp arrives last for that
-// (request, kv head) merges all its partials (wait-free: nobody ever waits for another warp).
+// whole context the warp normalises and writes the bf16 output rows itself.  Otherwise its fp32
+// partial (m, l, O) waits in shared memory until the span has been streamed and is then merged in
+// two stages, both wait-free (nobody ever waits for another warp; whoever arrives last does the
+// work): the warps of a CTA that hold pieces of one (request, kv head) count themselves in on a
+// shared-memory counter and the last one folds their partials; if the pair continues in other CTAs
+// the folded result goes to global memory as the CTA's one partial of it, an arrival counter in
+// global memory is bumped, and the last CTA to arrive merges the CTAs' partials.
 // ------------------------------------------------------------------------------------------
 struct AttnParams {
     const int32_t *block_tables;
@@ -508,7 +512,7 @@ struct AttnParams {
     const uint4 *k_new;             // bf16 [batch][Hkv][d]
     const uint4 *v_new;
     uint4 *pool_layer;
-    float *part_acc;                // [2*kMaxSpans][8][D]
+    float *part_acc;                // [2*kMaxSpans][8][D]   two slots per CTA are used: 2*cta, 2*cta + 1
     float *part_ml;                 // [2*kMaxSpans][16]  (m[8], l[8])
     int32_t *arrivals;              // [kMaxSpans], all zero between launches
     int4 *span_start;               // [kMaxSpans] what each span started at (diagnostic)

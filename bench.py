@@ -402,6 +402,7 @@ def run_ours(args) -> None:
             del dw
             torch.cuda.empty_cache()
             line["other_workloads"] = run_other_workloads(dev)
+            line["cuda_graph"] = run_cuda_graph(dev)
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(HEADLINE)
     if rank == 0:
@@ -522,6 +523,46 @@ def run_other_workloads(dev) -> list:
         del dw
         torch.cuda.empty_cache()
     return rows
+
+
+def run_cuda_graph(dev) -> dict:
+    """Launch overhead: 32 back-to-back steps issued call by call against the same 32 steps captured
+    once in a CUDA graph and replayed, on small and large batches of the mixed workload."""
+    import torch
+    rows = []
+    stream = torch.cuda.Stream(device=dev)
+    for b in (1, 8, 64):
+        dw = DeviceWorkload("mixed_sweep", dev, batch=b)
+        n, reps = 32, 20
+        try:
+            with torch.cuda.stream(stream):
+                dw.run_steps(n)
+                stream.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(reps):
+                    dw.run_steps(n)
+                e1.record(stream)
+                stream.synchronize()
+                eager_us = e0.elapsed_time(e1) * 1e3 / (n * reps)
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=stream):
+                    dw.run_steps(n)
+                graph.replay()
+                stream.synchronize()
+                e0.record(stream)
+                for _ in range(reps):
+                    graph.replay()
+                e1.record(stream)
+                stream.synchronize()
+                graph_us = e0.elapsed_time(e1) * 1e3 / (n * reps)
+            dw.kp.check_status()
+            rows.append({"batch": b, "eager_us_per_step": round(eager_us, 2), "graph_us_per_step": round(graph_us, 2)})
+        except Exception as exc:                      # capture not possible here: report, do not fail the bench
+            rows.append({"batch": b, "unavailable": str(exc)[:200]})
+        dw.kp.close()
+        del dw
+    return {"workload": "mixed_sweep", "steps_per_graph": 32, "points": rows}
 
 
 def run_autoscaler(sweep: dict) -> dict:

@@ -1173,26 +1173,33 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                     if (i & 1) mx1 = fmaxf(mx1, t); else mx0 = fmaxf(mx0, t);
                 }
             }
+            // The reference a column's exponentials are taken against only has to be near its maximum:
+            // it moves (with the reduction across lanes and the rescale that this costs) only when
+            // some score of the tile exceeds it by more than 2^8.
+            float mn0 = m0, mn1 = m1;
+            if (__any_sync(0xffffffffu, mx0 > m0 + 8.f || mx1 > m1 + 8.f)) {
 #pragma unroll
-            for (int x = 4; x < 32; x <<= 1) {
-                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, x));
-                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, x));
-            }
-            const float mo0 = m0, mo1 = m1;
-            float mn0 = fmaxf(mo0, mx0), mn1 = fmaxf(mo1, mx1);
-            m0 = mn0; m1 = mn1;
-            // a column that has seen no token yet (possible only for a later tile of a multi-token
-            // step) keeps m = -inf; exponentials are then taken against 0 so that they come out 0
-            if (kMulti) {
+                for (int x = 4; x < 32; x <<= 1) {
+                    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, x));
+                    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, x));
+                }
+                const float mo0 = m0, mo1 = m1;
+                mn0 = fmaxf(mo0, mx0); mn1 = fmaxf(mo1, mx1);
+                m0 = mn0; m1 = mn1;
+                if (kMulti) {
+                    mn0 = (mn0 == -INFINITY) ? 0.f : mn0;
+                    mn1 = (mn1 == -INFINITY) ? 0.f : mn1;
+                }
+                const float al0 = fast_exp2(mo0 - mn0), al1 = fast_exp2(mo1 - mn1);
+                l0 *= al0; l1 *= al1;
+#pragma unroll
+                for (int dt = 0; dt < Lay::kDTiles; ++dt) {
+                    o[dt][0] *= al0; o[dt][2] *= al0;
+                    o[dt][1] *= al1; o[dt][3] *= al1;
+                }
+            } else if (kMulti) {
                 mn0 = (mn0 == -INFINITY) ? 0.f : mn0;
                 mn1 = (mn1 == -INFINITY) ? 0.f : mn1;
-            }
-            const float al0 = fast_exp2(mo0 - mn0), al1 = fast_exp2(mo1 - mn1);
-            l0 *= al0; l1 *= al1;
-#pragma unroll
-            for (int dt = 0; dt < Lay::kDTiles; ++dt) {
-                o[dt][0] *= al0; o[dt][2] *= al0;
-                o[dt][1] *= al1; o[dt][3] *= al1;
             }
             uint32_t pb[kPagesPerTile][2];
 #pragma unroll

@@ -356,6 +356,21 @@ def run_ours(args) -> None:
                 "isolated": {"us_per_launch": attn_ms / attn_n * 1e3, "achieved": isolated, "frac": isolated / peak,
                              "timing": "events around every launch, no overlap between launches"}}
 
+    # ---- the read probe: the same tiles through the same rings, no arithmetic: the practical ceiling
+    def probe_steps(n):
+        for _ in range(n):
+            for layer in range(w.num_layers):
+                dw.kp.read_probe(layer, dw.bt, dw.sl)
+    probe_steps(W)
+    probe_ms, _ = timed_region(lambda: probe_steps(min(K, 500)), world, dev.index or 0)
+    dw.kp.check_status()
+    probe_us = probe_ms * 1e3 / (min(K, 500) * w.num_layers)
+    probe_gbs = (dw.bytes["kv"] // w.num_layers) / (probe_us * 1e-6) / 1e9
+    roofline["read_probe"] = {"us_per_launch": probe_us, "kv_gbs": probe_gbs,
+                              "attention_kv_gbs": (dw.bytes["kv"] // w.num_layers) / (us_launch * 1e-6) / 1e9,
+                              "frac_of_probe": probe_us / us_launch,
+                              "what": "kv_read_probe: the attention kernel's loads without its arithmetic, back to back"}
+
     # ---- end to end through the host-buffer entry point (pinned memory, copies inside the timing)
     E = min(K, 500)
     pin = lambda t: t.cpu().pin_memory()

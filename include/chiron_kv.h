@@ -172,6 +172,18 @@ int32_t decode_attention_multi(ckv_pool *pool, int32_t layer, int32_t batch, int
 int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *stream,
                     int32_t *h_header, int32_t *h_span_start);
 
+/*
+ * Read probe: streams exactly the KV tiles that decode_attention would read for this batch -- same
+ * partition, same TMA boxes, same ring depth per warp -- and does nothing with them.  Its running
+ * time is the practical ceiling of the memory system for this access pattern, which bench.py
+ * reports beside the attention kernel ("self-attention computation" being the part of the
+ * iteration that grows with the batch, Section 2.3, what bounds it is worth knowing).  Writes no
+ * output; bad page ids are flagged in the status word as in decode_attention.
+ * Errors: CKV_EINVAL, CKV_ECUDA.
+ */
+int32_t kv_read_probe(ckv_pool *pool, int32_t layer, int32_t batch,
+                      const int32_t *d_block_tables, const int32_t *d_seq_lens, void *stream);
+
 /* Number of spans the partition is balanced over (default: warps per CTA x number of SMs).
  * Setting it changes only how the context is split, never the result beyond fp32 summation
  * order.  1 <= num_spans <= 2048.  Errors: CKV_EINVAL. */

@@ -26,7 +26,7 @@ EXPORTS = (
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
     "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace", "ckv_set_overlap",
     "decode_attention_noalloc", "decode_step", "kv_swap_out", "kv_swap_in",
-    "kv_append_multi", "decode_attention_multi",
+    "kv_append_multi", "decode_attention_multi", "kv_read_probe",
     "local_autoscaler_instance_slo", "local_autoscaler_create", "local_autoscaler_destroy",
     "local_autoscaler_update", "local_autoscaler_get", "local_autoscaler_simulate",
     "global_request_groups", "global_waiting_time", "global_batch_backpressure", "global_batch_autoscale",
@@ -71,6 +71,7 @@ def _load() -> ctypes.CDLL:
     lib.kv_swap_in.restype = i32; lib.kv_swap_in.argtypes = [vp, i32, vp, vp, sz, vp]
     lib.kv_append_multi.restype = i32; lib.kv_append_multi.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.decode_attention_multi.restype = i32; lib.decode_attention_multi.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
+    lib.kv_read_probe.restype = i32; lib.kv_read_probe.argtypes = [vp, i32, i32, vp, vp, vp]
     lib.decode_plan.restype = i32; lib.decode_plan.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_set_partition.restype = i32; lib.ckv_set_partition.argtypes = [vp, i32]
     lib.ckv_set_overlap.restype = i32; lib.ckv_set_overlap.argtypes = [vp, i32]
@@ -240,6 +241,11 @@ class KvPool:
             raise ValueError("the swap image must be a contiguous pinned host tensor")
         _check(fn(self._h, int(page_ids.shape[0]), _dev_ptr(page_ids, torch.int32), image.data_ptr(),
                   image.numel() * image.element_size(), _stream_ptr(stream)))
+
+    def read_probe(self, layer: int, block_tables, seq_lens, stream=None) -> None:
+        """Stream the KV tiles decode_attention would read for this batch, without the arithmetic."""
+        _check(lib.kv_read_probe(self._h, layer, int(seq_lens.shape[0]), _dev_ptr(block_tables, torch.int32),
+                                 _dev_ptr(seq_lens, torch.int32), _stream_ptr(stream)))
 
     def decode_plan(self, seq_lens, stream=None):
         """(header dict, int32 [num_spans][4] array of span starts)."""

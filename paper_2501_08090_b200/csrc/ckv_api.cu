@@ -221,6 +221,17 @@ int32_t launch_attention_noalloc(const CUtensorMap &tmap, const ckv::AttnParams 
     return CKV_OK;
 }
 
+template <int D, int W, int NS>
+int32_t launch_read_probe(ckv_pool *pool, const ckv::ProbeParams &pp, cudaStream_t stream)
+{
+    using Lay = ckv::AttnLayout<D, W, NS>;
+    auto kernel = ckv::pool_read_probe_kernel<D, W, NS>;
+    CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
+    kernel<<<(pool->num_spans + W - 1) / W, W * 32, Lay::kSmemBytes, stream>>>(pool->tmap, pp);
+    CKV_CUDA(cudaGetLastError());
+    return CKV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -495,6 +506,31 @@ int32_t decode_step(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t 
     if (!d_k_new || !d_v_new) return fail(CKV_EINVAL, "decode_step: NULL k_new/v_new");
     return attention_launch(pool, "decode_step", layer, batch, 1, d_block_tables, d_seq_lens, d_q, d_k_new, d_v_new,
                             d_out, stream);
+}
+
+int32_t kv_read_probe(ckv_pool *pool, int32_t layer, int32_t batch, const int32_t *d_block_tables,
+                      const int32_t *d_seq_lens, void *stream)
+{
+    if (int32_t rc = check_call(pool, layer, batch, "kv_read_probe")) return rc;
+    if (!d_block_tables || !d_seq_lens) return fail(CKV_EINVAL, "kv_read_probe: NULL argument");
+    const ckv_config &c = pool->cfg;
+    ckv::ProbeParams pp{};
+    pp.block_tables = d_block_tables;
+    pp.seq_lens = d_seq_lens;
+    pp.status = pool->wsp<uint32_t>(pool->ws.status);
+    pp.sink = reinterpret_cast<unsigned long long *>(pool->d_ws + pool->ws.status + 64);
+    pp.batch = batch;
+    pp.max_pages_per_req = c.max_pages_per_req;
+    pp.num_pages = c.num_pages;
+    pp.num_kv_heads = c.num_kv_heads;
+    pp.layer_page_base = layer * c.num_pages;
+    pp.num_spans = pool->num_spans;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int32_t rc = c.head_dim == 128 ? launch_read_probe<128, kWarps128, kStages128>(pool, pp, s)
+                                         : launch_read_probe<64, kWarps64, kStages64>(pool, pp, s);
+    if (rc) return rc;
+    pool->launches += 1;
+    return CKV_OK;
 }
 
 int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, void *stream,

@@ -1521,4 +1521,83 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// Read probe: the attention kernel's loads without its arithmetic.  Every warp takes the same span
+// of the same plan, fetches the same tiles with the same TMA boxes through a ring of the same
+// depth, and only waits for them to land.  What this kernel takes is what the memory system gives
+// this access pattern: the practical ceiling the attention kernel is measured against.
+// ------------------------------------------------------------------------------------------
+struct ProbeParams {
+    const int32_t *block_tables;
+    const int32_t *seq_lens;
+    uint32_t *status;
+    unsigned long long *sink;       // receives a checksum of a few loaded words so that the loads count
+    int32_t batch, max_pages_per_req, num_pages, num_kv_heads;
+    int32_t layer_page_base, num_spans;
+};
+
+template <int D, int W, int NS>
+__global__ void __launch_bounds__(W * 32, 1)
+pool_read_probe_kernel(const __grid_constant__ CUtensorMap tmap, const ProbeParams p)
+{
+    using Lay = AttnLayout<D, W, NS>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int span = blockIdx.x * W + warp;
+    if (span >= p.num_spans) return;
+    const uint32_t ring = smem_u32(smem) + warp * NS * Lay::kStageBytes;
+    const uint32_t bars = smem_u32(smem + Lay::kBarOff) + warp * NS * 8;
+    if (lane == 0) {
+        prefetch_tensormap(&tmap);
+        for (int s = 0; s < NS; ++s) mbar_init(bars + s * 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    __syncwarp();
+    const SpanStart st = warp_plan(p.seq_lens, p.batch, p.max_pages_per_req, p.num_kv_heads, p.num_spans, span, lane);
+    if (st.r < 0) return;
+    AttnParams ap{};                              // the cursor reads only these
+    ap.seq_lens = p.seq_lens; ap.batch = p.batch; ap.max_pages_per_req = p.max_pages_per_req;
+    ap.num_kv_heads = p.num_kv_heads; ap.q_len = 1;
+    const uint64_t policy = l2_evict_first_policy();
+    SpanCursor ic;
+    ic.r = st.r; ic.h = st.h; ic.tile = st.tile; ic.L = st.L; ic.tiles = st.tiles_r; ic.v = st.v;
+    bool more = true;
+    int issued = 0, done = 0;
+    auto issue = [&]() {
+        const int n_pages = (ic.L + kPageSize - 1) / kPageSize;
+        const int np = min(kPagesPerTile, n_pages - ic.tile * kPagesPerTile);
+        const int pg = lane / Lay::kHalves, hf = lane % Lay::kHalves;
+        const int slot = issued % NS;
+        if (lane == 0) mbar_arrive_expect_tx(bars + slot * 8, np * Lay::kPageBytes);
+        __syncwarp();
+        if (lane < np * Lay::kHalves) {
+            int page = __ldg(p.block_tables + (size_t)ic.r * p.max_pages_per_req + ic.tile * kPagesPerTile + pg);
+            if (page < 0 || page >= p.num_pages) { atomicOr(p.status, kStatusBadPage); page = 0; }
+            const int y = ((p.layer_page_base + page) * p.num_kv_heads + ic.h) * 32;
+            tma_load_2d(ring + slot * Lay::kStageBytes + pg * Lay::kPageBytes + hf * Lay::kHalfBytes, &tmap, hf * 64, y,
+                        bars + slot * 8, policy);
+        }
+        ++issued;
+        more = ic.next(ap) && ic.v < st.end;
+    };
+    for (int k = 0; k < NS && more; ++k) issue();
+    uint32_t acc = 0;
+    bool alive = true;
+    while (done < issued) {
+        // every copy issued is waited for (each wait bounded), also after one of them gave up
+        const bool ok = mbar_wait_bounded(bars + (done % NS) * 8, (done / NS) & 1, p.status);
+        if (!__all_sync(0xffffffffu, ok)) alive = false;
+        if (alive) {
+            uint32_t v;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(ring + (done % NS) * Lay::kStageBytes + lane * 4));
+            acc ^= v;
+        }
+        ++done;
+        if (more && alive) issue();
+    }
+    if (acc == 0x9e3779b9u && lane == 0) atomicAdd(p.sink, 1ull);     // keeps the loads alive; practically never taken
+}
+
 }  // namespace ckv

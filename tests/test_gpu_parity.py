@@ -306,6 +306,24 @@ def test_attention_kernel_derives_the_same_partition_as_the_plan():
     assert ds.pool.check_status() == 0
 
 
+def test_read_probe_streams_the_batch_and_reports_bad_pages():
+    b = binding()
+    h = custom_inputs([700, 90, 2000, 64, 1500, 333, 800, 16, 5000], 8, 2, 128, seed=73)
+    ds = make_device_step(h)
+    before = dev_to_bits(ds.pool.pool).copy()
+    for C in (ds.pool.get_partition(), 5, 2048):
+        ds.pool.set_partition(C)
+        n0 = ds.pool.launch_count()
+        ds.pool.read_probe(0, ds.bt, ds.sl)
+        assert ds.pool.launch_count() - n0 == 1
+        assert ds.pool.check_status() == 0
+    assert np.array_equal(dev_to_bits(ds.pool.pool), before)              # a probe writes nothing
+    bad = ds.bt.clone()
+    bad[2, 3] = h.num_pages + 5
+    ds.pool.read_probe(0, bad, ds.sl)
+    assert ds.pool.check_status(raise_on_error=False) & b.STATUS_BAD_PAGE
+
+
 # --------------------------------------------------------------------------- merge stages
 
 @pytest.mark.parametrize("Hq,Hkv", [(4, 1), (8, 1), (8, 2)])

@@ -197,11 +197,21 @@ int32_t ckv_get_partition(const ckv_pool *pool);
  * they must not be produced by the kernel that immediately precedes decode_attention in the
  * stream (tables copied by a memcpy, or written by any earlier kernel, are fine -- the usual case,
  * since a serving engine uploads them once per iteration).  decode_step, being the only writer of
- * its layer's pool, also starts its first KV tile loads before that wait: with overlap on, a
- * kernel of the CALLER's that immediately precedes decode_step must not write pool pages that
- * this step reads.  The library's own writers are taken care of: after kv_append,
- * kv_append_multi or kv_swap_in on this handle the next decode_step waits before its loads, and
- * a preceding decode_step's appended rows are replaced in this step's staged tiles anyway.
+ * its layer's pool, also starts its first KV tile loads before that wait -- but never a tile that
+ * holds position seq_lens[r]-2 or later of its (request, KV head).  Position seq_lens[r]-1 is this
+ * step's own row (patched into the staged tile, whatever the copy saw); position seq_lens[r]-2 is
+ * what the previous decode_step of a loop that grows every context by one token per step stored,
+ * and that kernel may still be running.  Every kernel of this library releases its successor only
+ * after its own wait, so the early loads overlap the immediately preceding kernel and nothing
+ * older.  What follows for callers with overlap on:
+ *   - a kernel of the CALLER's that immediately precedes decode_step must not write pool pages
+ *     that this step reads;
+ *   - if the immediately preceding kernel is a decode_step on the same layer, each request of this
+ *     step must have grown by at most one token since (the same lengths replayed, as a benchmark
+ *     does, are fine too); an engine that rewrites older positions in place calls kv_append or
+ *     turns overlap off.
+ * The library's other writers are taken care of: after kv_append, kv_append_multi or kv_swap_in
+ * on this handle the next decode_step keeps all its loads behind the wait.
  * Turning overlap off restores plain stream order.  Errors: CKV_EINVAL. */
 int32_t ckv_set_overlap(ckv_pool *pool, int32_t enable);
 

@@ -78,10 +78,10 @@ struct AppendParams {
 
 __global__ void kv_append_kernel(const AppendParams p)
 {
-    // The pool may still be read by the attention kernel launched before this one: let the next
-    // kernel start its prologue, then wait for the predecessor before the first write.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // The pool may still be read by the attention kernel launched before this one: wait for the
+    // predecessor before the first write, then let the next kernel start its prologue.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int vec_per_row = p.head_dim / 8;                       // 16-byte pieces per row
     const int per_tok = p.num_kv_heads * 2 * vec_per_row;
     const int per_req = per_tok * p.q_len;
@@ -861,7 +861,6 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     const uint32_t bars = smem_u32(smem + Lay::kBarOff) + warp * NS * 8;
     int *cta_ctr = (int *)(smem + Lay::kCtrOff);
 
-    grid_launch_dependents();
     if (threadIdx.x < W) cta_ctr[threadIdx.x] = 0;
     __syncthreads();                             // the only CTA-wide barrier: the counters of the CTA stage are zero
     if (span >= p.num_spans) return;
@@ -882,6 +881,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                                    p.q_len);
     if (st.r < 0 || span == 0) {
         grid_dependency_wait();
+        grid_launch_dependents();
         if (span == 0)
             flag_unusable_requests(p.seq_lens, p.batch, p.max_pages_per_req, p.q_len, lane, p.out,
                                    p.q_len * p.num_q_heads * D, p.status);
@@ -1007,24 +1007,29 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 #endif
     };
 
-    // A step with the fused append is the only writer of its layer's pool, and what it computes does
-    // not depend on whether a tile's copy saw this step's new rows (they are put into the staged
-    // tile before use).  Its first loads can therefore start before the preceding kernel has
-    // finished -- under that kernel's tail -- as long as nothing of q, k_new or v_new is touched yet.
+    // A step with the fused append is the only writer of its layer's pool, so its first loads can
+    // start before the preceding kernel has finished -- under that kernel's tail -- as long as
+    // nothing of q, k_new or v_new is touched yet and no tile is fetched that the preceding kernel
+    // may still be writing.  If that kernel is the previous decode step of this layer, it writes
+    // each request's previous last position, L-2 as seen from this step (this step's own row, L-1,
+    // is put into the staged tile before use, so its copy may race with the store).  Tiles that
+    // hold a position >= L-2 therefore stay behind the dependency wait.  The dependents of this
+    // kernel are released only after the wait, so a kernel's early loads overlap its immediate
+    // predecessor and nothing older.
     const bool early = p.k_new != nullptr && p.early_loads != 0;
     if (early) {
         inputs_ready = false;
-        for (int k = 0; k < NS && more_to_issue; ++k) issue_next();
+        while (issued < NS && more_to_issue && ic.tile < (ic.L - 2) / kTileTokens) issue_next();
         inputs_ready = true;
     }
     grid_dependency_wait();                       // the workspace, q, the new rows and `out` are ours from here on
+    grid_launch_dependents();
     if (lane == 0) {
         p.span_start[span] = make_int4(st.r, st.h, st.tile, (int)st.v);
         p.trace[span * 8 + 0] = t_start;
         p.trace[span * 8 + 1] = 0;
     }
-    if (!early)
-        for (int k = 0; k < NS && more_to_issue; ++k) issue_next();
+    while (issued < NS && more_to_issue) issue_next();
 
     // ---- compute side
     SpanCursor cc;

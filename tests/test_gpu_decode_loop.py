@@ -93,3 +93,55 @@ def test_randomized_shapes_lengths_and_partitions():
             assert np.array_equal(dev_to_bits(kp.pool), ref_pool), what
             assert_close(dev_to_bits(out), ref, what)
             kp.close()
+
+
+def test_fused_loop_at_full_size_with_poisoned_future_slots():
+    """The decode loop at the 8B shape, batch 64: 72 fused steps enqueued behind one another with
+    no synchronisation, every context growing by one token per step.  Every slot that no step has
+    written yet -- and every unused page -- holds bf16 NaN, so a tile copy that read a row before
+    the preceding step's store of it landed shows up as a NaN output row instead of hiding inside
+    the tolerance.  All outputs must be finite; every step is compared with the oracle, and so is
+    the final pool, byte for byte."""
+    from paper_2501_08090_b200 import binding as b
+    w = wl.workload("llama8b_b64")
+    steps, B, Hq, Hkv, d = 72, w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim
+    start = wl.seq_lens(w) - 1                                             # lengths before the first step
+    # a few contexts that cross a tile boundary (multiple of 32) early in the loop
+    start[:4] = [1023, 2047 - 3, 511 + 17, 4000]
+    final = start + steps
+    npg = int(wl.pages_of(final).sum()) + 64
+    bt = wl.block_tables(final, npg, seed=5)
+    sh = PoolShape(1, npg, Hq, Hkv, 16, d)
+    pool_h = np.full(sh.elems, 0x7FC0, dtype=np.uint16)                    # NaN everywhere ...
+    view = pool_h.reshape(npg, Hkv, 2, 16, d)
+    for r in range(B):                                                     # ... except the tokens that exist
+        pos = np.arange(int(start[r]))
+        view[bt[r, pos // 16], :, :, pos % 16, :] = wl.normal_bf16((pos.size, Hkv, 2, d), 91, 100 + r)
+    q_h = wl.normal_bf16((steps, B, Hq, d), 91, 2)
+    k_h = wl.normal_bf16((steps, B, Hkv, d), 91, 3)
+    v_h = wl.normal_bf16((steps, B, Hkv, d), 91, 4)
+
+    cfg = b.make_config(1, Hq, Hkv, d, npg, bt.shape[1], B)
+    kp = b.KvPool(cfg, pool=bits_to_dev(pool_h))
+    btd = torch.from_numpy(bt).cuda()
+    lens_d = torch.from_numpy(np.stack([start + s + 1 for s in range(steps)]).astype(np.int32)).cuda()
+    q, k, v = bits_to_dev(q_h), bits_to_dev(k_h), bits_to_dev(v_h)
+    out = torch.full_like(q, float("nan"))
+    hold = torch.empty(1 << 28, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    for _ in range(4):
+        hold.fill_(1)                                                      # the launches below queue up behind this
+    for s in range(steps):
+        kp.decode_step(0, btd, lens_d[s], q[s], k[s], v[s], out[s])
+    assert kp.check_status() == 0
+    got = dev_to_bits(out)
+    assert np.all(np.isfinite(wl.bf16_bits_to_f32(got))), "a step read a slot before its store landed"
+
+    ref_pool = pool_h.copy()
+    for s in range(steps):
+        lens = (start + s + 1).astype(np.int32)
+        assert oracle.kv_append(ref_pool, sh, 0, bt, lens, k_h[s], v_h[s]) == 0
+        ref = oracle.decode_attention(ref_pool, sh, 0, bt, lens, q_h[s])
+        assert_close(got[s], ref, "step %d" % s)
+    assert np.array_equal(dev_to_bits(kp.pool), ref_pool)
+    kp.close()

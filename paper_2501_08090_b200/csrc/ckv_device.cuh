@@ -20,7 +20,6 @@ constexpr int kTileTokens = kPageSize * kPagesPerTile;
 constexpr int kMaxGroup = 8;         // query heads per KV head handled by one MMA column block
 constexpr int kMaxSpans = 2048;      // upper bound on the partition width (one span per warp)
 constexpr int kMaxBatch = 8192;
-constexpr int kBulkMergeFrom = 4;    // merges of more partials than this go through shared memory
 constexpr int kTreeFrom = 24;        // pairs cut into more partials than this are merged in two levels
 
 constexpr uint32_t kStatusBadLength = 1u;
@@ -535,268 +534,199 @@ struct AttnParams {
 // Output rows of a (request, kv head) start at out_rows (new token q_base); column c's row is
 // out_rows + (c / G) * qi_stride + (c % G) * D.
 //
-// Merge the partials of one (request, kv head) that spans s_first..s_last hold, and write its bf16
-// output rows.  Run by one whole warp (the last one to arrive for that pair).  Loads are issued in
-// batches so the merge costs a few L2 round trips, not one per partial.
+// ---- the fold: ONE routine merges partials, wherever they come from ------------------------
 //
-// Which partials: numbers i0, i0 + stride, ... (`pieces` of them) of the pair, where partial i lives
-// in slot_first (i = 0) or in the first slot of span s_first + i.  Where the result goes: to
-// dst_acc / dst_ml as one merged partial (same format, not normalised) if dst_acc is not NULL,
-// else normalised to the bf16 output rows.
-struct MergeSel {
-    int s_first, slot_first;   // the pair's first span and the slot of its partial 0
-    int i0, stride, pieces;    // the partials to merge
+// A partial is the triple (m, l, O) of a (request, kv head) over part of its context: m[8] the
+// reference the exponentials were taken against (log2 domain), l[8] their sums, O[8][D] the
+// weighted value sums, one row per column.  In memory it is `rows` (ncp rows of D floats at some
+// pitch) plus 16 floats (m[8], l[8]).  ncp is the live column count rounded up to a power of two
+// (at least 128 / D), so that the ncp * D floats of the rows split evenly over the 32 lanes: lane
+// owns 4 * J consecutive floats of ONE row g (J = ncp * D / 128 float4 pieces starting at
+// element d0).  A lane therefore needs one factor per partial, not eight, and the code below has
+// no per-column unrolling: it is small, which matters because every warp runs it once, after its
+// span, from an instruction cache that has held nothing but the streaming loop.
+//
+// Folding n partials in a fixed order t = 0 .. n-1:  M = max m_t, f_t = 2^(m_t - M),
+// L = sum f_t l_t, O = sum f_t O_t, in rounds of at most `cap` partials with the running (M, L, O)
+// rescaled when a round raises M.  The result is either normalised (O / L) to the bf16 output
+// rows or stored as one partial again.  The order of summation depends only on t, never on which
+// warp does the work, so results are bit-identical from run to run.
+struct FoldGeom {
+    int ncp, J, g, d0;
+};
+
+__device__ __forceinline__ FoldGeom fold_geometry(int ncols, int D, int lane)
+{
+    FoldGeom fg;
+    int ncp = 128 / D;                           // D = 64: at least two rows, so a lane owns a whole float4
+    while (ncp < ncols) ncp *= 2;
+    fg.ncp = ncp;
+    fg.J = ncp * D / 128;
+    fg.g = lane * ncp / 32;
+    fg.d0 = (lane * 4 * fg.J) % D;
+    return fg;
+}
+
+struct FoldJob {
+    int n;                          // partials to fold, in this order
+    int cap;                        // partials per round (shared-memory sources: n)
+    // partial t of a round that starts at t0 sits in shared memory at base + (t - t0) * stride:
+    // rows of `pitch` floats, (m, l) at byte offset ml_off ...
+    uint32_t base;
+    int stride, pitch, ml_off;
+    // ... except partial alt_t (if >= 0), which sits at alt_base
+    int alt_t;
+    uint32_t alt_base;
+    int alt_pitch, alt_ml_off;
+    // fetch != 0: the partials are in global memory -- number i0 + t * istride of a (request, kv
+    // head) whose partial 0 is slot slot_first and whose partial i > 0 is slot 2 * (s_first + i) --
+    // and are brought to `base` by bulk copies counted on mbarrier `bar` (phases used so far: uses)
+    int fetch, s_first, slot_first, i0, istride;
+    uint32_t bar;
+    int uses;
+    // destination: normalised bf16 rows if out_rows != NULL; else global partial slot dst_slot and,
+    // if copy_base != 0, the same partial once more in shared memory
+    uint16_t *out_rows;
+    int dst_slot;
+    uint32_t copy_base;
+    int copy_pitch, copy_ml_off;
+
     __device__ __forceinline__ int slot_of(int t) const
     {
-        const int i = i0 + t * stride;
+        const int i = i0 + t * istride;
         return i == 0 ? slot_first : 2 * (s_first + i);
     }
 };
 
-template <int D>
-__device__ __forceinline__ void store_merged(const float4 (&acc)[kMaxGroup], const float (&mstar)[kMaxGroup],
-                                             const float (&lsum)[kMaxGroup], float *dst_acc, float *dst_ml,
-                                             uint16_t *out_rows, int ncols, int G, int qi_stride, int lane)
+struct FoldCtx {
+    float *part_acc;                // [slots][8][D]
+    float *part_ml;                 // [slots][16]
+    uint32_t *status;
+    int ncols, G, qi_stride, lane;
+    FoldGeom fg;
+};
+
+__device__ __forceinline__ float ld_shared_f32(uint32_t addr)
 {
-#pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g) {
-        if (dst_acc != nullptr) {
-            if (g < ncols && lane * 4 < D) *(float4 *)(dst_acc + g * D + lane * 4) = acc[g];
-            if (lane == 0) { dst_ml[g] = mstar[g]; dst_ml[kMaxGroup + g] = lsum[g]; }
-        } else if (g < ncols && lane * 4 < D) {
-            const float inv = 1.f / lsum[g];
-            uint2 packed;
-            packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
-            packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
-            *(uint2 *)(out_rows + (size_t)(g / G) * qi_stride + (size_t)(g % G) * D + lane * 4) = packed;
-        }
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+
+// Start the bulk copies of one round (partials t0 .. t0 + cnt - 1) of a job with global sources.
+template <int D>
+__device__ __noinline__ void fold_fetch(const FoldJob j, const FoldCtx c, int t0)
+{
+    const int cnt = min(j.cap, j.n - t0);
+    const int row_bytes = c.fg.ncp * D * 4;
+    const bool alt_here = j.alt_t >= t0 && j.alt_t < t0 + cnt;
+    if (c.lane == 0) mbar_arrive_expect_tx(j.bar, (cnt - (alt_here ? 1 : 0)) * (row_bytes + 64));
+    __syncwarp();
+    if (c.lane < cnt && t0 + c.lane != j.alt_t) {
+        const int slot = j.slot_of(t0 + c.lane);
+        const uint32_t dst = j.base + c.lane * j.stride;
+        bulk_load_1d(dst, c.part_acc + (size_t)slot * kMaxGroup * D, row_bytes, j.bar);
+        bulk_load_1d(dst + j.ml_off, c.part_ml + slot * 2 * kMaxGroup, 64, j.bar);
     }
 }
 
+// Fold a job and store its result.  With global sources the first round's copies are already on
+// their way (fold_fetch).  Returns the number of phases the job's mbarrier has completed, or -1 if
+// a bounded wait gave up (nothing is stored then).
 template <int D>
-__device__ __noinline__ void combine_partials(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
-                                              uint16_t *out_rows, const MergeSel sel, float *dst_acc, float *dst_ml,
-                                              int ncols, int G, int qi_stride, int lane)
+__device__ __noinline__ int fold_finish(const FoldJob j, const FoldCtx c)
 {
-    const int pieces = sel.pieces;
-    auto slot_of = [&](int t) { return sel.slot_of(t); };
-
-    // (m, l) of the partial this lane owns in the first round of 32; usually the only round
-    float mi[kMaxGroup], li[kMaxGroup];
-    auto load_ml = [&](int i) {
-        const float *ml = part_ml + slot_of(i) * 2 * kMaxGroup;
-        const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
-        const float4 c = ld_cg_f32x4(ml + 8), d = ld_cg_f32x4(ml + 12);
-        mi[0] = a.x; mi[1] = a.y; mi[2] = a.z; mi[3] = a.w; mi[4] = b.x; mi[5] = b.y; mi[6] = b.z; mi[7] = b.w;
-        li[0] = c.x; li[1] = c.y; li[2] = c.z; li[3] = c.w; li[4] = d.x; li[5] = d.y; li[6] = d.z; li[7] = d.w;
-    };
-    float mstar[kMaxGroup];
+    const int g = c.fg.g, d0 = c.fg.d0, J = c.fg.J;
+    float M = -INFINITY, L = 0.f;
+    float4 acc[8];
 #pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g) mstar[g] = -INFINITY;
-    for (int base = (pieces - 1) & ~31; base >= 0; base -= 32) {       // chunk 0 last: its values stay in mi, li
-        if (base + lane < pieces) {
-            load_ml(base + lane);
-#pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g) mstar[g] = fmaxf(mstar[g], mi[g]);
-        }
-    }
-#pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g)
-#pragma unroll
-        for (int x = 16; x > 0; x >>= 1) mstar[g] = fmaxf(mstar[g], __shfl_xor_sync(0xffffffffu, mstar[g], x));
-
-    float lsum[kMaxGroup];
-    float4 acc[kMaxGroup];
-#pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g) { lsum[g] = 0.f; acc[g] = make_float4(0.f, 0.f, 0.f, 0.f); }
-    for (int base = 0; base < pieces; base += 32) {
-        // lane i of this round owns piece base + i: its factors and its share of the row sums
-        float f_mine[kMaxGroup];
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g) f_mine[g] = 0.f;
-        if (base + lane < pieces) {
-            if (base > 0) load_ml(base + lane);
-#pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g) {
-                // a column may have seen no token in any of these partials (a group of a multi-token
-                // step's two-level merge): its maximum stays -inf and its factors are 0
-                f_mine[g] = fast_exp2(mi[g] - (mstar[g] == -INFINITY ? 0.f : mstar[g]));
-                lsum[g] += f_mine[g] * li[g];
+    for (int q = 0; q < 8; ++q) acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+    int uses = j.uses;
+#pragma unroll 1
+    for (int t0 = 0; t0 < j.n; t0 += j.cap) {
+        const int cnt = min(j.cap, j.n - t0);
+        if (j.fetch) {
+            if (t0 > 0) {
+                fence_proxy_async();             // the last round's reads precede this round's copies
+                __syncwarp();
+                fold_fetch<D>(j, c, t0);
             }
+            bool ok = mbar_wait_bounded(j.bar, uses & 1, c.status);
+            ok = __all_sync(0xffffffffu, ok);
+            ++uses;
+            if (!ok) return -1;
         }
-        const int cnt = min(32, pieces - base);
-#pragma unroll 2
+        float Mr = -INFINITY;
+#pragma unroll 1
         for (int i = 0; i < cnt; ++i) {
-            const float *pa = part_acc + (size_t)slot_of(base + i) * kMaxGroup * D + lane * 4;
-#pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g) {
-                const float f = __shfl_sync(0xffffffffu, f_mine[g], i);
-                if (g < ncols && lane * 4 < D) {
-                    const float4 a = ld_cg_f32x4(pa + g * D);
-                    acc[g].x += f * a.x; acc[g].y += f * a.y; acc[g].z += f * a.z; acc[g].w += f * a.w;
-                }
-            }
+            const uint32_t ml = (t0 + i == j.alt_t) ? j.alt_base + j.alt_ml_off : j.base + i * j.stride + j.ml_off;
+            Mr = fmaxf(Mr, ld_shared_f32(ml + 4 * g));
         }
-    }
+        // a column that no partial so far has seen a token for keeps -inf (multi-token steps):
+        // exponentials are then taken against 0 and come out 0
+        const float Mn = fmaxf(M, Mr);
+        const float ref = Mn == -INFINITY ? 0.f : Mn;
+        const float sc = fast_exp2(M - ref);
+        M = Mn;
+        L *= sc;
 #pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g) {
-#pragma unroll
-        for (int x = 16; x > 0; x >>= 1) lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], x);
-    }
-    store_merged<D>(acc, mstar, lsum, dst_acc, dst_ml, out_rows, ncols, G, qi_stride, lane);
-}
-
-// Merge of up to two (request, kv head) pairs with at most four partials each -- the usual case at
-// large batch, where a warp's first and last piece each pair up with a neighbour.  Lanes 0..3 own
-// the partials of pair 0, lanes 4..7 those of pair 1; every accumulator load of both pairs is
-// issued before any of them is needed, so the whole merge costs about one memory round trip.
-template <int D>
-__device__ __noinline__ void combine_small_pairs(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
-                                                 int n_pairs, int first0, int last0, int slot0, uint16_t *out0,
-                                                 int first1, int last1, int slot1, uint16_t *out1, int ncols, int G,
-                                                 int qi_stride, int lane)
-{
-    const int pair = (lane >> 2) & 1, pi = lane & 3;
-    const int my_first = pair ? first1 : first0, my_last = pair ? last1 : last0, my_slot0 = pair ? slot1 : slot0;
-    const bool mine = lane < 8 && pair < n_pairs && pi <= my_last - my_first;
-    float mi[kMaxGroup], li[kMaxGroup];
-#pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g) { mi[g] = -INFINITY; li[g] = 0.f; }
-    if (mine) {
-        const int slot = pi == 0 ? my_slot0 : 2 * (my_first + pi);
-        const float *ml = part_ml + slot * 2 * kMaxGroup;
-        const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
-        const float4 c = ld_cg_f32x4(ml + 8), d = ld_cg_f32x4(ml + 12);
-        mi[0] = a.x; mi[1] = a.y; mi[2] = a.z; mi[3] = a.w; mi[4] = b.x; mi[5] = b.y; mi[6] = b.z; mi[7] = b.w;
-        li[0] = c.x; li[1] = c.y; li[2] = c.z; li[3] = c.w; li[4] = d.x; li[5] = d.y; li[6] = d.z; li[7] = d.w;
-    }
-    float f_mine[kMaxGroup], lsum[kMaxGroup];
-#pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g) {                       // reductions stay inside each group of four lanes
-        float mx = fmaxf(mi[g], __shfl_xor_sync(0xffffffffu, mi[g], 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        f_mine[g] = mine ? fast_exp2(mi[g] - mx) : 0.f;
-        float ls = f_mine[g] * li[g];
-        ls += __shfl_xor_sync(0xffffffffu, ls, 1);
-        ls += __shfl_xor_sync(0xffffffffu, ls, 2);
-        lsum[g] = ls;
-    }
-#pragma unroll
-    for (int it = 0; it < 2; ++it) {
-        if (it >= n_pairs) break;
-        const int f0 = it ? first1 : first0, pieces = (it ? last1 : last0) - f0 + 1, s0 = it ? slot1 : slot0;
-        uint16_t *out_rows = it ? out1 : out0;
-        float4 acc[kMaxGroup];
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g) acc[g] = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (i >= pieces) break;
-            const int slot = i == 0 ? s0 : 2 * (f0 + i);
-            const float *pa = part_acc + (size_t)slot * kMaxGroup * D + lane * 4;
-#pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g) {
-                const float f = __shfl_sync(0xffffffffu, f_mine[g], it * 4 + i);
-                if (g < ncols && lane * 4 < D) {
-                    const float4 a = ld_cg_f32x4(pa + g * D);
-                    acc[g].x += f * a.x; acc[g].y += f * a.y; acc[g].z += f * a.z; acc[g].w += f * a.w;
-                }
-            }
-        }
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g) {
-            const float lg = __shfl_sync(0xffffffffu, lsum[g], it * 4);
-            if (g < ncols && lane * 4 < D) {
-                const float inv = 1.f / lg;
-                uint2 packed;
-                packed.x = pack_bf16x2(acc[g].x * inv, acc[g].y * inv);
-                packed.y = pack_bf16x2(acc[g].z * inv, acc[g].w * inv);
-                *(uint2 *)(out_rows + (size_t)(g / G) * qi_stride + (size_t)(g % G) * D + lane * 4) = packed;
-            }
-        }
-    }
-}
-
-// The same merge for (request, kv head) pairs cut into many partials (small batches, very long
-// contexts): the partial accumulators are fetched with bulk async copies into the warp's ring --
-// idle once its span has been streamed -- up to `cap` partials per round, and summed from shared
-// memory.  A round costs one copy latency however many partials it holds.  `uses` counts how many
-// phases the mbarrier `bar` has completed so far and is advanced here.  Returns false if a
-// bounded wait gave up.
-template <int D>
-__device__ __noinline__ bool combine_partials_bulk(const float *__restrict__ part_acc, const float *__restrict__ part_ml,
-                                                   uint16_t *out_rows, const MergeSel sel, float *dst_acc, float *dst_ml,
-                                                   int ncols, int G, int qi_stride, int lane, uint32_t ring, int ring_bytes,
-                                                   uint32_t bar, int &uses, uint32_t *status)
-{
-    const int pieces = sel.pieces;
-    auto slot_of = [&](int t) { return sel.slot_of(t); };
-    const int piece_bytes = ncols * D * 4;                   // the live rows of a partial are contiguous
-    const int cap = min(32, ring_bytes / piece_bytes);
-
-    // running maximum over the rounds seen so far; sums are rescaled when it grows (online merge),
-    // so no separate pass over the (m, l) rows is needed
-    float mstar[kMaxGroup], lsum[kMaxGroup];
-    float4 acc[kMaxGroup];
-#pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g) { mstar[g] = -INFINITY; lsum[g] = 0.f; acc[g] = make_float4(0.f, 0.f, 0.f, 0.f); }
-    bool ok = true;
-    for (int base = 0; base < pieces && ok; base += cap) {
-        const int cnt = min(cap, pieces - base);
-        if (lane == 0) mbar_arrive_expect_tx(bar, cnt * piece_bytes);
-        __syncwarp();
-        float mi[kMaxGroup], li[kMaxGroup];
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g) { mi[g] = -INFINITY; li[g] = 0.f; }
-        if (lane < cnt) {                                     // lane i owns partial base + i of this round
-            const int slot = slot_of(base + lane);
-            bulk_load_1d(ring + lane * piece_bytes, part_acc + (size_t)slot * kMaxGroup * D, piece_bytes, bar);
-            const float *ml = part_ml + slot * 2 * kMaxGroup;
-            const float4 a = ld_cg_f32x4(ml), b = ld_cg_f32x4(ml + 4);
-            const float4 c = ld_cg_f32x4(ml + 8), d = ld_cg_f32x4(ml + 12);
-            mi[0] = a.x; mi[1] = a.y; mi[2] = a.z; mi[3] = a.w; mi[4] = b.x; mi[5] = b.y; mi[6] = b.z; mi[7] = b.w;
-            li[0] = c.x; li[1] = c.y; li[2] = c.z; li[3] = c.w; li[4] = d.x; li[5] = d.y; li[6] = d.z; li[7] = d.w;
-        }
-        float f_mine[kMaxGroup];
-#pragma unroll
-        for (int g = 0; g < kMaxGroup; ++g) {
-            float mx = mi[g];
-#pragma unroll
-            for (int x = 16; x > 0; x >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, x));
-            const float mnew = fmaxf(mstar[g], mx);
-            // -inf only while no partial so far has seen a token for this column (a multi-token step):
-            // exponentials are then taken against 0 and come out 0
-            const float mref = mnew == -INFINITY ? 0.f : mnew;
-            const float rescale = fast_exp2(mstar[g] - mref);
-            mstar[g] = mnew;
-            acc[g].x *= rescale; acc[g].y *= rescale; acc[g].z *= rescale; acc[g].w *= rescale;
-            f_mine[g] = fast_exp2(mi[g] - mref);              // lanes without a partial: exp2(-inf) = 0
-            lsum[g] = lsum[g] * rescale + f_mine[g] * li[g];
-        }
-        ok = mbar_wait_bounded(bar, uses & 1, status);
-        ok = __all_sync(0xffffffffu, ok);
-        ++uses;
-        if (!ok) break;
+        for (int q = 0; q < 8; ++q) { acc[q].x *= sc; acc[q].y *= sc; acc[q].z *= sc; acc[q].w *= sc; }
+#pragma unroll 1
         for (int i = 0; i < cnt; ++i) {
+            const bool alt = t0 + i == j.alt_t;
+            const uint32_t pb = alt ? j.alt_base : j.base + i * j.stride;
+            const uint32_t ml = pb + (alt ? j.alt_ml_off : j.ml_off);
+            const uint32_t rows = pb + (g * (alt ? j.alt_pitch : j.pitch) + d0) * 4;
+            const float f = fast_exp2(ld_shared_f32(ml + 4 * g) - ref);
+            L += f * ld_shared_f32(ml + 4 * (kMaxGroup + g));
 #pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g) {
-                const float f = __shfl_sync(0xffffffffu, f_mine[g], i);
-                if (g < ncols && lane * 4 < D) {
-                    const float4 a = ld_shared_f32x4(ring + i * piece_bytes + g * D * 4 + lane * 16);
-                    acc[g].x += f * a.x; acc[g].y += f * a.y; acc[g].z += f * a.z; acc[g].w += f * a.w;
+            for (int q = 0; q < 8; ++q) {
+                if (q < J) {
+                    const float4 a = ld_shared_f32x4(rows + q * 16);
+                    acc[q].x += f * a.x; acc[q].y += f * a.y; acc[q].z += f * a.z; acc[q].w += f * a.w;
                 }
             }
         }
-        __syncwarp();                                         // all reads of this round precede the next round's copies
+        __syncwarp();                            // every lane has read the round before anything overwrites it
     }
-    if (!ok) return false;
+    if (j.out_rows != nullptr) {
+        if (g < c.ncols) {
+            const float inv = 1.f / L;
+            uint16_t *row = j.out_rows + (size_t)(g / c.G) * c.qi_stride + (size_t)(g % c.G) * D + d0;
 #pragma unroll
-    for (int g = 0; g < kMaxGroup; ++g) {
+            for (int q = 0; q < 8; ++q) {
+                if (q < J) {
+                    uint2 packed;
+                    packed.x = pack_bf16x2(acc[q].x * inv, acc[q].y * inv);
+                    packed.y = pack_bf16x2(acc[q].z * inv, acc[q].w * inv);
+                    *(uint2 *)(row + q * 4) = packed;
+                }
+            }
+        }
+    } else {
+        float *rows = c.part_acc + (size_t)j.dst_slot * kMaxGroup * D + g * D + d0;
 #pragma unroll
-        for (int x = 16; x > 0; x >>= 1) lsum[g] += __shfl_xor_sync(0xffffffffu, lsum[g], x);
+        for (int q = 0; q < 8; ++q)
+            if (q < J) *(float4 *)(rows + q * 4) = acc[q];
+        if (d0 == 0) {
+            c.part_ml[j.dst_slot * 2 * kMaxGroup + g] = M;
+            c.part_ml[j.dst_slot * 2 * kMaxGroup + kMaxGroup + g] = L;
+        }
+        if (j.copy_base != 0) {
+            const uint32_t crow = j.copy_base + (g * j.copy_pitch + d0) * 4;
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (q < J)
+                    asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(crow + q * 16), "f"(acc[q].x), "f"(acc[q].y),
+                                 "f"(acc[q].z), "f"(acc[q].w) : "memory");
+            if (d0 == 0) {
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(j.copy_base + j.copy_ml_off + 4 * g), "f"(M) : "memory");
+                asm volatile("st.shared.f32 [%0], %1;" ::"r"(j.copy_base + j.copy_ml_off + 4 * (kMaxGroup + g)), "f"(L) : "memory");
+            }
+            __syncwarp();
+        }
     }
-    store_merged<D>(acc, mstar, lsum, dst_acc, dst_ml, out_rows, ncols, G, qi_stride, lane);
-    return true;
+    return uses;
 }
 
 template <int D, int W, int NS>
@@ -1056,7 +986,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     int n_pieces = 0;
     bool first_piece = true;
     // a span writes at most two partials: its first piece and its last piece
-    int pend_first[2] = {-1, -1}, pend_last[2] = {0, 0}, pend_slot[2] = {0, 0};
+    int pend_first[2] = {-1, -1}, pend_last[2] = {0, 0};
     uint16_t *pend_out[2] = {nullptr, nullptr};
     while (more_to_compute) {
         const int n = (int)min((long long)(cc.tiles - cc.tile), v_end - cc.v);
@@ -1276,7 +1206,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             if (entered) {
 #pragma unroll
                 for (int g = 0; g < kMaxGroup; ++g)
-                    if (g < ncols && lane * 4 < D)
+                    if (lane * 4 < D)
                         *(float4 *)(park + g * D + lane * 4) = *(const float4 *)(staging + g * Lay::kStagePitch + lane * 4);
             }
             if (lane < 4) {
@@ -1302,19 +1232,48 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
 
     if (lane == 0) p.trace[span * 8 + 2] = global_timer_ns();
 
-    // ---- CTA stage.  Consecutive spans belong to the warps of one CTA, so the partials of a
-    // (request, kv head) that several of this CTA's warps hold are merged through shared memory:
-    // each warp counts itself in on a shared counter once its span has been streamed, and the last
-    // one folds the CTA's partials (wait-free, no global round trip).  If the pair lies inside this
-    // CTA the result is final; otherwise it is the CTA's one partial of the pair for the grid stage.
+    // ---- hand-over.  Every merge below is one FoldJob run by fold_finish.
+    //
+    // CTA stage: consecutive spans belong to the warps of one CTA, so the partials of a (request,
+    // kv head) that several of this CTA's warps hold are folded straight from shared memory: each
+    // warp counts itself in on a shared counter once its span has been streamed, and the last one
+    // does the fold (wait-free, no global round trip).  If the pair lies inside this CTA the result
+    // is final; otherwise it is the CTA's one partial of the pair: it goes to global memory and,
+    // once more, into this warp's own buffer.
+    // Grid stage, in units of CTAs: the CTA that arrives last for a pair (a counter in global
+    // memory) fetches the other CTAs' partials into its idle ring with bulk copies and folds them
+    // with its own; a pair cut into more than kTreeFrom partials is folded in two levels.
+    FoldCtx fc;
+    fc.part_acc = p.part_acc; fc.part_ml = p.part_ml; fc.status = p.status;
+    fc.ncols = ncols; fc.G = G; fc.qi_stride = qi_stride; fc.lane = lane;
+    fc.fg = fold_geometry(ncols, D, lane);
+    const uint32_t staging_u32 = smem_u32(smem + Lay::kStagingOff), park_u32 = smem_u32(smem + Lay::kParkOff);
+    constexpr int kStagingMl = kMaxGroup * Lay::kStagePitch * 4, kParkMl = kMaxGroup * D * 4;
+    const int part_bytes = fc.fg.ncp * D * 4 + 64;               // a fetched partial in the ring: rows, then (m, l)
+    int bar_uses[2] = {(done + NS - 1) / NS, (done + NS - 2) / NS};   // phases the first two stage barriers have completed
+    FoldJob jobs[2];
+    int n_jobs = 0;
+    int tree_first[2] = {-1, -1}, tree_last[2] = {0, 0};         // pairs that take the counter protocol for more than two CTAs
+    uint16_t *tree_out[2] = {nullptr, nullptr};
+    uint32_t tree_buf[2] = {0u, 0u};
+    auto grid_job = [&](int c_first, int n, int i0, int istride, int alt_t, uint32_t buf, bool in_staging) {
+        FoldJob j;
+        j.n = n; j.cap = 1;                       // the ring region and cap are set when the jobs are started
+        j.base = 0; j.stride = part_bytes; j.pitch = D; j.ml_off = part_bytes - 64;
+        j.alt_t = alt_t; j.alt_base = buf;
+        j.alt_pitch = in_staging ? Lay::kStagePitch : D; j.alt_ml_off = in_staging ? kStagingMl : kParkMl;
+        j.fetch = 1; j.s_first = c_first; j.slot_first = 2 * c_first + 1; j.i0 = i0; j.istride = istride;
+        j.bar = 0; j.uses = 0;
+        j.out_rows = nullptr; j.dst_slot = 0; j.copy_base = 0; j.copy_pitch = 0; j.copy_ml_off = 0;
+        return j;
+    };
     {
         const int b0 = blockIdx.x * W;
-#pragma unroll 1                                      // executed once per warp: keep the code small, it runs from a cold instruction cache
-        for (int k = 0; k < 2; ++k) {
+#pragma unroll 1                                      // executed once per warp: keep the code small
+        for (int k = 0; k < 2 && alive; ++k) {
             if (pend_first[k] < 0) continue;
             const int f = pend_first[k], l = pend_last[k];
             const int fb = max(f, b0), lb = min(l, b0 + W - 1), cb = lb - fb + 1;
-            pend_first[k] = -1;                   // becomes a grid-stage entry below, if one is needed
             if (cb > 1) {
                 __threadfence_block();
                 __syncwarp();
@@ -1324,111 +1283,66 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 if (prior != cb - 1) continue;    // a later warp of this CTA folds them
                 __threadfence_block();
             }
-            // fold the partials of spans fb..lb: span f keeps its own in its staging tile, the others
+            // the partials of spans fb..lb: span f keeps its own in its staging tile, the others
             // (which the pair entered from the left) in their parking buffers
-            float mstar[kMaxGroup], lsum[kMaxGroup];
-            float4 acc[kMaxGroup];
-#pragma unroll
-            for (int g = 0; g < kMaxGroup; ++g) { mstar[g] = -INFINITY; lsum[g] = 0.f; acc[g] = make_float4(0.f, 0.f, 0.f, 0.f); }
-            auto rows_of = [&](int sp, int &pitch) -> const float * {
-                const int w = sp - b0;
-                if (sp == f) { pitch = Lay::kStagePitch; return (const float *)(smem + Lay::kStagingOff + w * Lay::kStagingBytes); }
-                pitch = D;
-                return (const float *)(smem + Lay::kParkOff + w * Lay::kParkBytes);
-            };
-            for (int sp = fb; sp <= lb; ++sp) {
-                int pitch;
-                const float *rows = rows_of(sp, pitch);
-                const float *ml = rows + kMaxGroup * pitch;
-#pragma unroll
-                for (int g = 0; g < kMaxGroup; ++g) mstar[g] = fmaxf(mstar[g], ml[g]);
-            }
-            for (int sp = fb; sp <= lb; ++sp) {
-                int pitch;
-                const float *rows = rows_of(sp, pitch);
-                const float *ml = rows + kMaxGroup * pitch;
-#pragma unroll
-                for (int g = 0; g < kMaxGroup; ++g) {
-                    // a column that has seen no token anywhere (multi-token step) keeps -inf: factors 0
-                    const float fct = fast_exp2(ml[g] - (mstar[g] == -INFINITY ? 0.f : mstar[g]));
-                    lsum[g] += fct * ml[kMaxGroup + g];
-                    if (g < ncols && lane * 4 < D) {
-                        const float4 a = *(const float4 *)(rows + g * pitch + lane * 4);
-                        acc[g].x += fct * a.x; acc[g].y += fct * a.y; acc[g].z += fct * a.z; acc[g].w += fct * a.w;
-                    }
-                }
-            }
+            const uint32_t my_buf = k == 0 ? park_u32 + warp * Lay::kParkBytes : staging_u32 + warp * Lay::kStagingBytes;
+            FoldJob j;
+            j.n = cb; j.cap = cb;
+            j.base = park_u32 + (fb - b0) * Lay::kParkBytes; j.stride = Lay::kParkBytes; j.pitch = D; j.ml_off = kParkMl;
+            j.alt_t = f >= fb ? 0 : -1;
+            j.alt_base = staging_u32 + (fb - b0) * Lay::kStagingBytes; j.alt_pitch = Lay::kStagePitch; j.alt_ml_off = kStagingMl;
+            j.fetch = 0; j.s_first = 0; j.slot_first = 0; j.i0 = 0; j.istride = 1; j.bar = 0; j.uses = 0;
+            j.out_rows = nullptr; j.dst_slot = 0; j.copy_base = 0; j.copy_pitch = 0; j.copy_ml_off = 0;
             const int c_first = f / W, c_last = l / W;
             if (c_first == c_last) {              // the pair lies inside this CTA: done
-                store_merged<D>(acc, mstar, lsum, nullptr, nullptr, pend_out[k], ncols, G, qi_stride, lane);
+                j.out_rows = pend_out[k];
+                fold_finish<D>(j, fc);
                 continue;
             }
             // partial 0 of a pair (the CTA it begins in) lives in that CTA's odd slot, the others in
             // the even slot of their CTA
-            const int slot = (int)blockIdx.x == c_first ? 2 * (int)blockIdx.x + 1 : 2 * (int)blockIdx.x;
-            // publish this CTA's partial; the stores drain while the counter is asked
-            store_merged<D>(acc, mstar, lsum, p.part_acc + (size_t)slot * kMaxGroup * D, p.part_ml + slot * 2 * kMaxGroup,
-                            nullptr, ncols, G, qi_stride, lane);
+            j.dst_slot = (int)blockIdx.x == c_first ? 2 * (int)blockIdx.x + 1 : 2 * (int)blockIdx.x;
+            if (cb > 1) {                         // keep the folded partial here as well
+                j.copy_base = my_buf;
+                j.copy_pitch = k == 0 ? D : Lay::kStagePitch;
+                j.copy_ml_off = k == 0 ? kParkMl : kStagingMl;
+            }
+            fold_finish<D>(j, fc);                // publish; the stores drain while the counter is asked
             if (c_last == c_first + 1) {
                 // Two CTAs share the pair.  If the other one has arrived already (counter at 1), its
-                // partial is published and this warp is the last: it merges straight from its
-                // registers -- one round trip for the counter, one for the other partial.  If not,
-                // it counts itself in; should the other one have arrived in between, it is the last
-                // after all and does the same.
+                // partial is published and this warp is the last.  If not, it counts itself in;
+                // should the other one have arrived in between, it is the last after all.
                 int seen = 0;
                 if (lane == 0) seen = atomicCAS(p.arrivals + c_first, 1, 0);
                 seen = __shfl_sync(0xffffffffu, seen, 0);
                 if (seen != 1) {
                     __threadfence();              // the partial's stores left before the counter was asked
+                    __syncwarp();
                     if (lane == 0) seen = atomicAdd(p.arrivals + c_first, 1);
                     seen = __shfl_sync(0xffffffffu, seen, 0);
                     if (seen != 1) continue;      // first to arrive: the other CTA merges
                     if (lane == 0) p.arrivals[c_first] = 0;
                 }
                 __threadfence();
-                const int other = (int)blockIdx.x == c_first ? 2 * c_last : 2 * c_first + 1;
-                const float *oml = p.part_ml + other * 2 * kMaxGroup;
-                const float *oacc = p.part_acc + (size_t)other * kMaxGroup * D + lane * 4;
-                const float4 m_lo = ld_cg_f32x4(oml), m_hi = ld_cg_f32x4(oml + 4);
-                const float4 l_lo = ld_cg_f32x4(oml + 8), l_hi = ld_cg_f32x4(oml + 12);
-                float4 oa[kMaxGroup];
-#pragma unroll
-                for (int g = 0; g < kMaxGroup; ++g)
-                    oa[g] = (g < ncols && lane * 4 < D) ? ld_cg_f32x4(oacc + g * D) : make_float4(0.f, 0.f, 0.f, 0.f);
-                const float om[kMaxGroup] = {m_lo.x, m_lo.y, m_lo.z, m_lo.w, m_hi.x, m_hi.y, m_hi.z, m_hi.w};
-                const float ol[kMaxGroup] = {l_lo.x, l_lo.y, l_lo.z, l_lo.w, l_hi.x, l_hi.y, l_hi.z, l_hi.w};
-#pragma unroll
-                for (int g = 0; g < kMaxGroup; ++g) {
-                    const float mx = fmaxf(mstar[g], om[g]);
-                    const float ref = mx == -INFINITY ? 0.f : mx;
-                    const float fa = fast_exp2(mstar[g] - ref), fo = fast_exp2(om[g] - ref);
-                    mstar[g] = mx;
-                    // products rounded separately, then added: the result is the same bits whichever
-                    // of the two CTAs does the merge
-                    lsum[g] = __fadd_rn(__fmul_rn(fa, lsum[g]), __fmul_rn(fo, ol[g]));
-                    acc[g].x = __fadd_rn(__fmul_rn(fa, acc[g].x), __fmul_rn(fo, oa[g].x));
-                    acc[g].y = __fadd_rn(__fmul_rn(fa, acc[g].y), __fmul_rn(fo, oa[g].y));
-                    acc[g].z = __fadd_rn(__fmul_rn(fa, acc[g].z), __fmul_rn(fo, oa[g].z));
-                    acc[g].w = __fadd_rn(__fmul_rn(fa, acc[g].w), __fmul_rn(fo, oa[g].w));
-                }
-                store_merged<D>(acc, mstar, lsum, nullptr, nullptr, pend_out[k], ncols, G, qi_stride, lane);
+                jobs[n_jobs] = grid_job(c_first, 2, 0, 1, (int)blockIdx.x - c_first, my_buf, k == 1);
+                jobs[n_jobs].out_rows = pend_out[k];
+                ++n_jobs;
                 continue;
             }
-            pend_first[k] = c_first; pend_last[k] = c_last; pend_slot[k] = 2 * c_first + 1;
+            tree_first[k] = c_first; tree_last[k] = c_last; tree_out[k] = pend_out[k]; tree_buf[k] = my_buf;
         }
     }
 
-    // ---- grid stage, in units of CTAs: whichever CTA arrives last for a (request, kv head) merges
-    // the CTAs' partials (wait-free).
-    if (pend_first[0] >= 0 || pend_first[1] >= 0) {
+    // ---- pairs shared by more than two CTAs: arrival counters
+    if (alive && (tree_first[0] >= 0 || tree_first[1] >= 0)) {
         int n_part[2], sub[2], grp[2], grp_cnt[2], n_grp[2];
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
-            n_part[k] = pend_first[k] >= 0 ? pend_last[k] - pend_first[k] + 1 : 0;
+            n_part[k] = tree_first[k] >= 0 ? tree_last[k] - tree_first[k] + 1 : 0;
             sub[k] = 0; grp[k] = 0; grp_cnt[k] = n_part[k]; n_grp[k] = 1;
             if (n_part[k] > kTreeFrom) {
                 sub[k] = merge_group_size(n_part[k]);
-                grp[k] = ((int)blockIdx.x - pend_first[k]) / sub[k];
+                grp[k] = ((int)blockIdx.x - tree_first[k]) / sub[k];
                 n_grp[k] = (n_part[k] + sub[k] - 1) / sub[k];
                 grp_cnt[k] = min(sub[k], n_part[k] - grp[k] * sub[k]);
             }
@@ -1437,71 +1351,71 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         __syncwarp();
         int prior0 = 0, prior1 = 0;
         if (lane == 0) {                          // both round trips in flight together
-            if (pend_first[0] >= 0) prior0 = atomicAdd(p.arrivals + pend_first[0] + (sub[0] ? 1 + grp[0] : 0), 1);
-            if (pend_first[1] >= 0) prior1 = atomicAdd(p.arrivals + pend_first[1] + (sub[1] ? 1 + grp[1] : 0), 1);
+            if (tree_first[0] >= 0) prior0 = atomicAdd(p.arrivals + tree_first[0] + (sub[0] ? 1 + grp[0] : 0), 1);
+            if (tree_first[1] >= 0) prior1 = atomicAdd(p.arrivals + tree_first[1] + (sub[1] ? 1 + grp[1] : 0), 1);
         }
         prior0 = __shfl_sync(0xffffffffu, prior0, 0);
         prior1 = __shfl_sync(0xffffffffu, prior1, 0);
         bool last[2];
-        last[0] = pend_first[0] >= 0 && prior0 == grp_cnt[0] - 1;
-        last[1] = pend_first[1] >= 0 && prior1 == grp_cnt[1] - 1;
+        last[0] = tree_first[0] >= 0 && prior0 == grp_cnt[0] - 1;
+        last[1] = tree_first[1] >= 0 && prior1 == grp_cnt[1] - 1;
         if (last[0] || last[1]) {
             __threadfence();
             if (lane == 0) {                      // counters are ready for the next launch
-                if (last[0]) p.arrivals[pend_first[0] + (sub[0] ? 1 + grp[0] : 0)] = 0;
-                if (last[1]) p.arrivals[pend_first[1] + (sub[1] ? 1 + grp[1] : 0)] = 0;
-            }
-            // stage 0's barrier has completed one phase per tile it carried; the ring is idle now
-            int bar_uses = (done + NS - 1) / NS;
-            auto merge = [&](int k, const MergeSel sel, float *dst_acc, float *dst_ml) {
-                if (alive && sel.pieces > kBulkMergeFrom) {
-                    fence_proxy_async();          // partials written through the generic proxy, read by bulk copies
-                    alive = combine_partials_bulk<D>(p.part_acc, p.part_ml, pend_out[k], sel, dst_acc, dst_ml, ncols, G,
-                                                     qi_stride, lane, ring, NS * Lay::kStageBytes, bars, bar_uses, p.status);
-                } else {
-                    combine_partials<D>(p.part_acc, p.part_ml, pend_out[k], sel, dst_acc, dst_ml, ncols, G, qi_stride, lane);
-                }
-            };
-            // first level of the two-level merges
-#pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                if (!last[k] || sub[k] == 0) continue;
-                MergeSel sel;
-                sel.s_first = pend_first[k]; sel.slot_first = pend_slot[k];
-                sel.i0 = grp[k] * sub[k]; sel.stride = 1; sel.pieces = grp_cnt[k];
-                const int dst_slot = sel.slot_of(0);
-                merge(k, sel, p.part_acc + (size_t)dst_slot * kMaxGroup * D, p.part_ml + dst_slot * 2 * kMaxGroup);
-                __threadfence();
-                __syncwarp();
-                int prior = 0;
-                if (lane == 0) prior = atomicAdd(p.arrivals + pend_first[k], 1);
-                prior = __shfl_sync(0xffffffffu, prior, 0);
-                last[k] = prior == n_grp[k] - 1;
-                if (last[k]) {
-                    __threadfence();
-                    if (lane == 0) p.arrivals[pend_first[k]] = 0;
-                }
-            }
-            // final merges
-            const int fin0 = last[0] ? (sub[0] ? n_grp[0] : n_part[0]) : 0;
-            const int fin1 = last[1] ? (sub[1] ? n_grp[1] : n_part[1]) : 0;
-            if ((last[0] || last[1]) && fin0 <= kBulkMergeFrom && fin1 <= kBulkMergeFrom && sub[0] == 0 && sub[1] == 0) {
-                // the usual case: one or two short merges, done together
-                const int a = last[0] ? 0 : 1, b = 1;
-                combine_small_pairs<D>(p.part_acc, p.part_ml, (last[0] ? 1 : 0) + (last[1] ? 1 : 0),
-                                       pend_first[a], pend_last[a], pend_slot[a], pend_out[a],
-                                       pend_first[b], pend_last[b], pend_slot[b], pend_out[b], ncols, G, qi_stride, lane);
-            } else {
-#pragma unroll
-                for (int k = 0; k < 2; ++k) {
-                    if (!last[k]) continue;
-                    MergeSel sel;
-                    sel.s_first = pend_first[k]; sel.slot_first = pend_slot[k];
-                    sel.i0 = 0; sel.stride = sub[k] ? sub[k] : 1; sel.pieces = k == 0 ? fin0 : fin1;
-                    merge(k, sel, nullptr, nullptr);
-                }
+                if (last[0]) p.arrivals[tree_first[0] + (sub[0] ? 1 + grp[0] : 0)] = 0;
+                if (last[1]) p.arrivals[tree_first[1] + (sub[1] ? 1 + grp[1] : 0)] = 0;
             }
         }
+#pragma unroll 1
+        for (int k = 0; k < 2 && alive; ++k) {
+            if (!last[k]) continue;
+            const int me = (int)blockIdx.x - tree_first[k];
+            if (sub[k] == 0) {                    // one level: this CTA's partial is still in its own buffer
+                jobs[n_jobs] = grid_job(tree_first[k], n_part[k], 0, 1, me, tree_buf[k], k == 1);
+                jobs[n_jobs].out_rows = tree_out[k];
+                ++n_jobs;
+                continue;
+            }
+            // first level of a two-level merge: fold this group's partials into the slot of its first
+            // member, right away and with the whole ring; then count the group in
+            FoldJob j = grid_job(tree_first[k], grp_cnt[k], grp[k] * sub[k], 1, me - grp[k] * sub[k], tree_buf[k], k == 1);
+            j.dst_slot = j.slot_of(0);
+            j.base = ring; j.cap = min(32, NS * Lay::kStageBytes / part_bytes);
+            j.bar = bars; j.uses = bar_uses[0];
+            fence_proxy_async();                  // partials written through the generic proxy, read by bulk copies
+            fold_fetch<D>(j, fc, 0);
+            const int u = fold_finish<D>(j, fc);
+            if (u < 0) { alive = false; break; }
+            bar_uses[0] = u;
+            __threadfence();
+            __syncwarp();
+            int prior = 0;
+            if (lane == 0) prior = atomicAdd(p.arrivals + tree_first[k], 1);
+            prior = __shfl_sync(0xffffffffu, prior, 0);
+            if (prior != n_grp[k] - 1) continue;
+            __threadfence();
+            if (lane == 0) p.arrivals[tree_first[k]] = 0;
+            jobs[n_jobs] = grid_job(tree_first[k], n_grp[k], 0, sub[k], -1, 0u, false);
+            jobs[n_jobs].out_rows = tree_out[k];
+            ++n_jobs;
+        }
+    }
+
+    // ---- run the grid-stage jobs: both fetches first, so that their round trips overlap
+    if (alive && n_jobs > 0) {
+        const int region = NS * Lay::kStageBytes / n_jobs;
+        fence_proxy_async();                      // partials written through the generic proxy, read by bulk copies
+#pragma unroll 1
+        for (int i = 0; i < n_jobs; ++i) {
+            jobs[i].base = ring + i * region;
+            jobs[i].cap = min(32, region / part_bytes);
+            jobs[i].bar = bars + i * 8;
+            jobs[i].uses = bar_uses[i];
+            fold_fetch<D>(jobs[i], fc, 0);
+        }
+#pragma unroll 1
+        for (int i = 0; i < n_jobs && alive; ++i)
+            if (fold_finish<D>(jobs[i], fc) < 0) alive = false;
     }
 
     // Do not leave while copies into this warp's ring may still be in flight (only after a wait gave up).

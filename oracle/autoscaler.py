@@ -15,11 +15,16 @@ The instance's ITL SLO is the smallest ITL SLO among the requests it runs.
 Readings where the text leaves room: BP exactly 1 halves (the algorithm's `< 1` test decides, not
 the prose's "greater than one"); MaxBS is kept as a real number clamped to [min_bs, max_bs]; the
 batch the instance actually runs is floor(MaxBS) capped by the demand; a zero current throughput
-counts as infinite backpressure.  TBP is the paper's test for "no throughput gain is observed from
-increasing the batch size" (Section 4.1), so the previous throughput is kept only across an update
-that INCREASED MaxBS; after a decrease (or at the start) there is none and TBP = 0.  Applied
-literally after a decrease, TBP would exceed one every time (throughput falls with the batch on
-the rising part of the curve) and each halving would trigger the next, down to a batch of one.
+counts as infinite backpressure.
+
+Which throughput is "previous".  Printed rule (`literal_tbp=True` below): the throughput observed
+at the update before, whatever that update did.  Default reading: Section 4.1 introduces TBP as
+the check on whether a larger batch still buys throughput, so the previous throughput is kept
+only across an update that INCREASED MaxBS; after a decrease (or at the start) there is none and
+TBP = 0.  The literal rule is unstable in closed loop: on the rising part of the curve a halving
+lowers the throughput, TBP reads above one at the next update, and each halving triggers the
+next, down to a batch of one.  Both are implemented here and in the library and tested side by
+side.
 """
 from __future__ import annotations
 
@@ -62,9 +67,16 @@ def interp_latency(batch_sizes: Sequence[float], us: Sequence[float], bs: float)
     raise AssertionError
 
 
+def next_baseline(thr: float, old_bs: float, new_bs: float, literal_tbp: bool) -> Optional[float]:
+    """The 'previous throughput' the NEXT update will compare against (None: no TBP term)."""
+    if literal_tbp or new_bs > old_bs:
+        return thr
+    return None
+
+
 def simulate(batch_sizes: Sequence[float], us: Sequence[float], extra_us: float, itl_slo_us: float,
              demand: int, initial_max_bs: float, iterations: int, alpha: float = 0.5,
-             min_bs: float = 1.0, max_cap: float = 1e9) -> List[Tuple[float, int, float, float]]:
+             min_bs: float = 1.0, max_cap: float = 1e9, literal_tbp: bool = False) -> List[Tuple[float, int, float, float]]:
     """Closed loop against a measured latency curve: rows of (MaxBS after the update, batch run,
     ITL in us, backpressure)."""
     max_bs, thr_prev, rows = float(initial_max_bs), None, []
@@ -74,7 +86,7 @@ def simulate(batch_sizes: Sequence[float], us: Sequence[float], extra_us: float,
         thr = bs / itl
         _, _, bp = backpressure(itl, itl_slo_us, thr_prev, thr)
         new_bs = update(max_bs, bp, alpha, min_bs, max_cap)
-        thr_prev = thr if new_bs > max_bs else None          # baseline only across an increase
+        thr_prev = next_baseline(thr, max_bs, new_bs, literal_tbp)
         max_bs = new_bs
         rows.append((max_bs, bs, itl, bp))
     return rows

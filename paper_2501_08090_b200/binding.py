@@ -30,7 +30,7 @@ EXPORTS = (
     "local_autoscaler_instance_slo", "local_autoscaler_create", "local_autoscaler_destroy",
     "local_autoscaler_update", "local_autoscaler_get", "local_autoscaler_simulate",
     "global_request_groups", "global_waiting_time", "global_batch_backpressure", "global_batch_autoscale",
-    "global_interactive_autoscale",
+    "global_interactive_autoscale", "global_autoscaler_simulate",
 )
 
 
@@ -42,7 +42,30 @@ class CkvError(RuntimeError):
 
 class AutoscalerConfig(ctypes.Structure):
     _fields_ = [("alpha", ctypes.c_double), ("itl_slo_us", ctypes.c_double),
-                ("min_bs", ctypes.c_double), ("max_bs", ctypes.c_double)]
+                ("min_bs", ctypes.c_double), ("max_bs", ctypes.c_double), ("tbp_mode", ctypes.c_int32)]
+
+
+class SimConfig(ctypes.Structure):
+    """ckv_sim_config of include/chiron_autoscaler.h."""
+    _fields_ = [("slots_interactive", ctypes.c_int32), ("slots_batch", ctypes.c_int32),
+                ("rate_interactive", ctypes.c_double), ("rate_batch", ctypes.c_double),
+                ("startup_s", ctypes.c_double), ("tick_s", ctypes.c_double),
+                ("theta", ctypes.c_double), ("delta", ctypes.c_double),
+                ("floor_instances", ctypes.c_int32), ("initial_instances", ctypes.c_int32),
+                ("max_batch_instances", ctypes.c_int32), ("groups_k", ctypes.c_int32),
+                ("z", ctypes.c_double), ("mu_o_prior", ctypes.c_double), ("sigma_o_prior", ctypes.c_double),
+                ("policy", ctypes.c_int32), ("horizon_s", ctypes.c_double)]
+
+
+class SimSummary(ctypes.Structure):
+    """ckv_sim_summary of include/chiron_autoscaler.h."""
+    _fields_ = [("end_s", ctypes.c_double), ("finished", ctypes.c_int32),
+                ("interactive_total", ctypes.c_int32), ("interactive_ttft_met", ctypes.c_int32),
+                ("batch_total", ctypes.c_int32), ("batch_ttft_met", ctypes.c_int32),
+                ("evictions", ctypes.c_int32),
+                ("instances_added", ctypes.c_int32 * 3), ("instances_removed", ctypes.c_int32 * 3),
+                ("instance_seconds", ctypes.c_double * 3), ("peak_instances", ctypes.c_int32 * 3),
+                ("tokens_served", ctypes.c_double)]
 
 
 class Config(ctypes.Structure):
@@ -103,6 +126,9 @@ def _load() -> ctypes.CDLL:
     lib.global_batch_autoscale.argtypes = [vp, vp, i32, f64, f64, f64, i32, i32, i32, f64, i32p]
     lib.global_interactive_autoscale.restype = i32
     lib.global_interactive_autoscale.argtypes = [i32, i32, f64, f64, i32, i32p]
+    lib.global_autoscaler_simulate.restype = i32
+    lib.global_autoscaler_simulate.argtypes = [ctypes.POINTER(SimConfig), i32, vp, vp, vp, vp, vp, vp, vp,
+                                               ctypes.POINTER(SimSummary), vp, vp, i32, ctypes.POINTER(i64)]
     lib.ckv_launch_count.restype = i64; lib.ckv_launch_count.argtypes = [vp]
     lib.ckv_last_error.restype = ctypes.c_char_p; lib.ckv_last_error.argtypes = []
     return lib
@@ -341,8 +367,8 @@ class LocalAutoscaler:
     """Per-instance batch-size autoscaler (Algorithm 1); host-only, thin wrapper over the C ABI."""
 
     def __init__(self, itl_slo_us: float, initial_max_bs: float, alpha: float = 0.5,
-                 min_bs: float = 1.0, max_bs: float = 1e9):
-        self.cfg = AutoscalerConfig(alpha, itl_slo_us, min_bs, max_bs)
+                 min_bs: float = 1.0, max_bs: float = 1e9, literal_tbp: bool = False):
+        self.cfg = AutoscalerConfig(alpha, itl_slo_us, min_bs, max_bs, 1 if literal_tbp else 0)
         self._h = ctypes.c_void_p()
         rc = lib.local_autoscaler_create(ctypes.byref(self.cfg), float(initial_max_bs), ctypes.byref(self._h))
         if rc != CKV_OK:
@@ -384,9 +410,10 @@ def instance_slo(itl_slos_us) -> float:
 
 
 def autoscaler_simulate(itl_slo_us: float, initial_max_bs: float, batch_sizes, us_per_step, extra_us: float,
-                        demand: int, iterations: int, alpha: float = 0.5, min_bs: float = 1.0, max_bs: float = 1e9):
+                        demand: int, iterations: int, alpha: float = 0.5, min_bs: float = 1.0, max_bs: float = 1e9,
+                        literal_tbp: bool = False):
     """Closed loop of Algorithm 1 over a latency curve: arrays (MaxBS, batch run, ITL us, backpressure)."""
-    cfg = AutoscalerConfig(alpha, itl_slo_us, min_bs, max_bs)
+    cfg = AutoscalerConfig(alpha, itl_slo_us, min_bs, max_bs, 1 if literal_tbp else 0)
     x = np.ascontiguousarray(batch_sizes, dtype=np.float64)
     y = np.ascontiguousarray(us_per_step, dtype=np.float64)
     o_bs = np.zeros(iterations, np.float64); o_b = np.zeros(iterations, np.int32)
@@ -447,3 +474,38 @@ def interactive_autoscale(busy: int, total: int, theta: float, delta: float, flo
     _rc(lib.global_interactive_autoscale(int(busy), int(total), float(theta), float(delta), int(floor),
                                          ctypes.byref(out)), "global_interactive_autoscale")
     return out.value
+
+
+SIM_POLICY_CHIRON, SIM_POLICY_IMMEDIATE = 0, 1
+SIM_EVENTS = ("ARRIVE", "START", "EVICT", "FINISH", "ADD", "READY", "REMOVE", "TICK")
+
+
+def global_simulate(cfg: SimConfig, arrival_s, kind, output_tokens, ttft_slo_s, log_cap: int = 0):
+    """Run the global autoscaler's discrete-event simulation (host-only).
+
+    Returns a dict: per-request arrays `first_start_s`, `finish_s`, `evictions`; `summary` (a plain
+    dict of ckv_sim_summary); `events` = number of events that occurred; and, if log_cap > 0,
+    `log` = list of (time, kind, a, b) rows (at most log_cap)."""
+    a = np.ascontiguousarray(arrival_s, dtype=np.float64)
+    k = np.ascontiguousarray(kind, dtype=np.int32)
+    o = np.ascontiguousarray(output_tokens, dtype=np.float64)
+    s = np.ascontiguousarray(ttft_slo_s, dtype=np.float64)
+    n = int(a.size)
+    if not (k.size == n and o.size == n and s.size == n):
+        raise ValueError("the four request arrays must have one entry per request")
+    first = np.zeros(n, np.float64); fin = np.zeros(n, np.float64); ev = np.zeros(n, np.int32)
+    summ = SimSummary()
+    lt = np.zeros(max(1, log_cap), np.float64); lr = np.zeros((max(1, log_cap), 3), np.int32)
+    rows = ctypes.c_int64(0)
+    rc = lib.global_autoscaler_simulate(ctypes.byref(cfg), n, a.ctypes.data, k.ctypes.data, o.ctypes.data,
+                                        s.ctypes.data, first.ctypes.data, fin.ctypes.data, ev.ctypes.data,
+                                        ctypes.byref(summ), lt.ctypes.data if log_cap else None,
+                                        lr.ctypes.data if log_cap else None, int(log_cap), ctypes.byref(rows))
+    _rc(rc, "global_autoscaler_simulate")
+    summary = {name: (list(getattr(summ, name)) if hasattr(getattr(summ, name), "__len__") else getattr(summ, name))
+               for name, _ in SimSummary._fields_}
+    out = {"first_start_s": first, "finish_s": fin, "evictions": ev, "summary": summary, "events": int(rows.value)}
+    if log_cap:
+        m = min(int(rows.value), log_cap)
+        out["log"] = [(float(lt[i]), int(lr[i, 0]), int(lr[i, 1]), int(lr[i, 2])) for i in range(m)]
+    return out

@@ -8,7 +8,8 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
-SOURCES = [os.path.join(CSRC, "ckv_api.cu"), os.path.join(CSRC, "ckv_autoscaler.cc")]
+SOURCES = [os.path.join(CSRC, "ckv_api.cu"), os.path.join(CSRC, "ckv_autoscaler.cc"),
+           os.path.join(CSRC, "ckv_global_sim.cc")]
 HEADERS = [os.path.join(CSRC, "ckv_device.cuh"), os.path.join(_ROOT, "include", "chiron_kv.h"),
            os.path.join(_ROOT, "include", "chiron_autoscaler.h")]
 LIBRARY = os.path.join(_HERE, "libchiron_kv.so")

@@ -12,7 +12,8 @@ constexpr int32_t kOk = 0, kInval = -1, kNoMem = -2;
 
 bool config_ok(const ckv_autoscaler_config *c)
 {
-    return c && c->alpha > 0.0 && c->alpha <= 1.0 && c->itl_slo_us > 0.0 && c->min_bs >= 1.0 && c->max_bs >= c->min_bs;
+    return c && c->alpha > 0.0 && c->alpha <= 1.0 && c->itl_slo_us > 0.0 && c->min_bs >= 1.0 && c->max_bs >= c->min_bs &&
+           (c->tbp_mode == CKV_TBP_AFTER_INCREASE || c->tbp_mode == CKV_TBP_LITERAL);
 }
 
 double clamp(double x, double lo, double hi) { return std::min(std::max(x, lo), hi); }
@@ -38,8 +39,9 @@ double step(ckv_autoscaler &a, double itl_us, double throughput, double *bp_out)
     else
         next = a.max_bs / 2.0;
     next = clamp(next, a.cfg.min_bs, a.cfg.max_bs);
-    // TBP asks whether the last INCREASE of the batch size paid off: keep the baseline only across one
-    a.has_prev = next > a.max_bs;
+    // default: TBP asks whether the last INCREASE of the batch size paid off, so the baseline is kept
+    // only across one; literal: the throughput of the update before, always
+    a.has_prev = a.cfg.tbp_mode == CKV_TBP_LITERAL || next > a.max_bs;
     a.prev_throughput = throughput;
     a.max_bs = next;
     if (bp_out) *bp_out = bp;

@@ -1307,33 +1307,16 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 j.copy_pitch = k == 0 ? D : Lay::kStagePitch;
                 j.copy_ml_off = k == 0 ? kParkMl : kStagingMl;
             }
-            fold_finish<D>(j, fc);                // publish; the stores drain while the counter is asked
-            if (c_last == c_first + 1) {
-                // Two CTAs share the pair.  If the other one has arrived already (counter at 1), its
-                // partial is published and this warp is the last.  If not, it counts itself in;
-                // should the other one have arrived in between, it is the last after all.
-                int seen = 0;
-                if (lane == 0) seen = atomicCAS(p.arrivals + c_first, 1, 0);
-                seen = __shfl_sync(0xffffffffu, seen, 0);
-                if (seen != 1) {
-                    __threadfence();              // the partial's stores left before the counter was asked
-                    __syncwarp();
-                    if (lane == 0) seen = atomicAdd(p.arrivals + c_first, 1);
-                    seen = __shfl_sync(0xffffffffu, seen, 0);
-                    if (seen != 1) continue;      // first to arrive: the other CTA merges
-                    if (lane == 0) p.arrivals[c_first] = 0;
-                }
-                __threadfence();
-                jobs[n_jobs] = grid_job(c_first, 2, 0, 1, (int)blockIdx.x - c_first, my_buf, k == 1);
-                jobs[n_jobs].out_rows = pend_out[k];
-                ++n_jobs;
-                continue;
-            }
+            fold_finish<D>(j, fc);                // publish: the stores drain while the counters are asked
             tree_first[k] = c_first; tree_last[k] = c_last; tree_out[k] = pend_out[k]; tree_buf[k] = my_buf;
         }
     }
 
-    // ---- pairs shared by more than two CTAs: arrival counters
+    // ---- arrival of this CTA's partials (both pairs together: two round trips in all).
+    // A pair shared by two CTAs first asks its counter with a compare-and-swap: if the other CTA has
+    // arrived already (counter at 1) this warp is the last and takes the counter back to 0 in the
+    // same operation.  The fence that publishes this warp's partials runs while those are in flight.
+    // Everybody else then counts itself in; whoever brings a counter to its full count is the last.
     if (alive && (tree_first[0] >= 0 || tree_first[1] >= 0)) {
         int n_part[2], sub[2], grp[2], grp_cnt[2], n_grp[2];
 #pragma unroll
@@ -1347,25 +1330,35 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 grp_cnt[k] = min(sub[k], n_part[k] - grp[k] * sub[k]);
             }
         }
-        __threadfence();
+        int seen0 = 0, seen1 = 0;
+        if (lane == 0) {
+            if (n_part[0] == 2) seen0 = atomicCAS(p.arrivals + tree_first[0], 1, 0);
+            if (n_part[1] == 2) seen1 = atomicCAS(p.arrivals + tree_first[1], 1, 0);
+        }
+        __threadfence();                          // the partials' stores have left; what the other CTAs published is visible
         __syncwarp();
-        int prior0 = 0, prior1 = 0;
+        seen0 = __shfl_sync(0xffffffffu, seen0, 0);
+        seen1 = __shfl_sync(0xffffffffu, seen1, 0);
+        bool last[2];
+        last[0] = n_part[0] == 2 && seen0 == 1;
+        last[1] = n_part[1] == 2 && seen1 == 1;
+        int prior0 = -1, prior1 = -1;
         if (lane == 0) {                          // both round trips in flight together
-            if (tree_first[0] >= 0) prior0 = atomicAdd(p.arrivals + tree_first[0] + (sub[0] ? 1 + grp[0] : 0), 1);
-            if (tree_first[1] >= 0) prior1 = atomicAdd(p.arrivals + tree_first[1] + (sub[1] ? 1 + grp[1] : 0), 1);
+            if (tree_first[0] >= 0 && !last[0]) prior0 = atomicAdd(p.arrivals + tree_first[0] + (sub[0] ? 1 + grp[0] : 0), 1);
+            if (tree_first[1] >= 0 && !last[1]) prior1 = atomicAdd(p.arrivals + tree_first[1] + (sub[1] ? 1 + grp[1] : 0), 1);
         }
         prior0 = __shfl_sync(0xffffffffu, prior0, 0);
         prior1 = __shfl_sync(0xffffffffu, prior1, 0);
-        bool last[2];
-        last[0] = tree_first[0] >= 0 && prior0 == grp_cnt[0] - 1;
-        last[1] = tree_first[1] >= 0 && prior1 == grp_cnt[1] - 1;
-        if (last[0] || last[1]) {
+        const bool late0 = prior0 >= 0 && prior0 == grp_cnt[0] - 1, late1 = prior1 >= 0 && prior1 == grp_cnt[1] - 1;
+        if (late0 || late1) {
             __threadfence();
             if (lane == 0) {                      // counters are ready for the next launch
-                if (last[0]) p.arrivals[tree_first[0] + (sub[0] ? 1 + grp[0] : 0)] = 0;
-                if (last[1]) p.arrivals[tree_first[1] + (sub[1] ? 1 + grp[1] : 0)] = 0;
+                if (late0) p.arrivals[tree_first[0] + (sub[0] ? 1 + grp[0] : 0)] = 0;
+                if (late1) p.arrivals[tree_first[1] + (sub[1] ? 1 + grp[1] : 0)] = 0;
             }
         }
+        last[0] = last[0] || late0;
+        last[1] = last[1] || late1;
 #pragma unroll 1
         for (int k = 0; k < 2 && alive; ++k) {
             if (!last[k]) continue;

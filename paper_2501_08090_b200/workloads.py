@@ -225,3 +225,35 @@ def algorithmic_bytes(w: Workload, lens: np.ndarray, num_layers: Optional[int] =
     tables = int(pages_of(lens, w.page_size).sum()) * 4 + b * 4
     return {"kv": layers * kv, "q_out": layers * qo, "append": layers * append,
             "tables": layers * tables, "total": layers * (kv + qo + append + tables)}
+
+
+# ----------------------------------------------------------------------------- request traces
+
+def arrival_times(n: int, rate: float, cv: float, seed: int, start: float = 0.0) -> np.ndarray:
+    """n arrival times with mean rate `rate` per second and inter-arrival coefficient of variation
+    `cv`: Gamma inter-arrivals of shape 1 / cv^2 (cv = 1 is a Poisson process, Section 6
+    "Workloads"; larger cv is burstier, Section 6 "Impact of Arrival Burstiness")."""
+    rng = np.random.default_rng([int(seed), 0xA221])
+    shape = 1.0 / (cv * cv)
+    gaps = rng.gamma(shape, 1.0 / (shape * rate), size=n)
+    return start + np.cumsum(gaps)
+
+
+def output_lengths(n: int, seed: int, median: float = 180.0, sigma: float = 0.9, cap: int = 2048) -> np.ndarray:
+    """Synthetic output-token counts: lognormal, clipped to [1, cap].  Stands in for the ShareGPT
+    output-length distribution the paper's traces use (not available offline)."""
+    rng = np.random.default_rng([int(seed), 0x0077])
+    return np.clip(np.rint(np.exp(math.log(median) + sigma * rng.standard_normal(n))), 1, cap)
+
+
+def request_trace(n: int, rate: float, cv: float, batch_fraction: float, seed: int,
+                  interactive_ttft_s: float = 10.0, batch_ttft_s: float = 3600.0):
+    """A trace of n requests in arrival order: (arrival_s, kind [0 interactive, 1 batch],
+    output_tokens, ttft_slo_s) with the paper's two request classes (Section 6 "Workloads":
+    interactive TTFT SLO 10 s, batch TTFT SLO one hour)."""
+    arrival = arrival_times(n, rate, cv, seed)
+    rng = np.random.default_rng([int(seed), 0x7A3C])
+    kind = (rng.random(n) < batch_fraction).astype(np.int32)
+    tokens = output_lengths(n, seed)
+    slo = np.where(kind == 0, interactive_ttft_s, batch_ttft_s).astype(np.float64)
+    return arrival, kind, tokens, slo

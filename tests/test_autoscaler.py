@@ -24,7 +24,7 @@ def cases():
     out = []
     for line in open(GOLDEN):
         line = line.strip()
-        if not line or line.startswith("#"):
+        if not line or line.startswith("#") or line.startswith("seq"):
             continue
         name, slo, bs, itl, tp, tc, bp, after = [x.strip() for x in line.split("|")]
         out.append((name, float(slo), float(bs), float(itl), None if tp == "-" else float(tp), float(tc),
@@ -81,6 +81,48 @@ def test_a_decrease_does_not_trigger_the_next_one(b):
     assert bp == pytest.approx(0.5) and bs == 48.0
     bs, bp = a.update(150.0, 500.0)                # now an increase is being judged: throughput fell 600 -> 500
     assert bp == pytest.approx(1.2) and bs == 24.0
+
+
+def two_update_cases():
+    out = []
+    for line in open(GOLDEN):
+        if line.startswith("seq"):
+            f = [x.strip() for x in line.split("|")]
+            out.append((f[1], *[float(x) for x in f[2:]]))
+    return out
+
+
+@pytest.mark.parametrize("case", two_update_cases(), ids=[c[0] for c in two_update_cases()])
+def test_the_two_readings_of_previous_throughput(b, case):
+    reading, slo, bs0, itl1, thr1, bs1, itl2, thr2, bp2, bs2 = case
+    literal = reading == "literal"
+    # the restatement
+    _, _, bp = ref.backpressure(itl1, slo, None, thr1)
+    after1 = ref.update(bs0, bp)
+    assert after1 == bs1
+    base = ref.next_baseline(thr1, bs0, after1, literal)
+    _, _, bp = ref.backpressure(itl2, slo, base, thr2)
+    assert bp == pytest.approx(bp2, rel=1e-12) and ref.update(after1, bp) == bs2
+    # the library
+    a = b.LocalAutoscaler(itl_slo_us=slo, initial_max_bs=bs0, literal_tbp=literal)
+    assert a.update(itl1, thr1)[0] == bs1
+    got_bs, got_bp = a.update(itl2, thr2)
+    assert got_bp == pytest.approx(bp2, rel=1e-12) and got_bs == bs2
+
+
+def test_literal_previous_throughput_collapses_in_closed_loop(b):
+    """On a curve whose throughput still rises with the batch, the literal TBP rule turns the first
+    halving into a cascade down to a batch of one and never recovers more than a step; the default
+    reading keeps probing the SLO point."""
+    sizes, us = linear_curve()
+    slo, extra = 1000.0, 200.0                                # ITL(bs) = 230 + 4 bs  ->  bs* = 192
+    lit = b.autoscaler_simulate(slo, 4.0, sizes, us, extra, demand=10000, iterations=400, literal_tbp=True)
+    want = ref.simulate(list(sizes), list(us), extra, slo, 10000, 4.0, 400, literal_tbp=True)
+    assert np.allclose(lit[0], [r[0] for r in want], rtol=1e-12)
+    dflt = b.autoscaler_simulate(slo, 4.0, sizes, us, extra, demand=10000, iterations=400)
+    assert lit[1][100:].min() == 1                            # the cascade reaches a batch of one ...
+    assert np.mean(lit[1][100:]) < 0.5 * np.mean(dflt[1][100:])   # ... and the loop serves far fewer requests per step
+    assert dflt[1][100:].min() >= 40                          # the default keeps probing between half the peak and the peak
 
 
 def test_instance_slo_is_the_smallest(b):

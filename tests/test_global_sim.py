@@ -1,0 +1,268 @@
+"""The global autoscaler as a discrete-event simulation (paper Section 3 life cycle, Section 5
+autoscaling): the library's C++ against a hand-worked event trace, event for event against the
+independently structured Python event loop in oracle/global_sim.py on seeded Poisson and Gamma
+traces, and against what the paper says the mechanism does (over-provisioning absorbs a spike of
+1/Theta, queueing instead of immediate scaling cuts hysteresis, no backpressure adds nothing,
+idle batch instances are retired)."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import global_sim as ref
+from paper_2501_08090_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "global_sim_trace.txt")
+KINDS = {"ARRIVE": 0, "START": 1, "EVICT": 2, "FINISH": 3, "ADD": 4, "READY": 5, "REMOVE": 6, "TICK": 7}
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2501_08090_b200 import build
+    build.build()
+    from paper_2501_08090_b200 import binding
+    return binding
+
+
+def base_config(**over):
+    kw = dict(slots_interactive=8, slots_batch=32, rate_interactive=20.0, rate_batch=8.0, startup_s=30.0, tick_s=5.0,
+              theta=1.0 / 3.0, delta=0.05, floor_instances=1, initial_instances=3, max_batch_instances=64,
+              groups_k=3, z=1.0, mu_o_prior=200.0, sigma_o_prior=150.0, policy=0, horizon_s=0.0)
+    kw.update(over)
+    return kw
+
+
+def run_both(b, kw, trace):
+    got = b.global_simulate(b.SimConfig(**kw), *trace, log_cap=2_000_000)
+    want = ref.simulate(ref.SimConfig(**kw), *trace)
+    return got, want
+
+
+def assert_same_run(got, want):
+    assert got["events"] == len(want.log)
+    for i, (x, y) in enumerate(zip(got["log"], want.log)):
+        assert x == y, "event %d differs: library %r, oracle %r" % (i, x, y)
+    s = want.summary()
+    for key, val in got["summary"].items():
+        if isinstance(val, list):
+            assert val == pytest.approx(s[key], rel=1e-12, abs=1e-9), key
+        else:
+            assert val == pytest.approx(s[key], rel=1e-12, abs=1e-9), key
+    assert np.array_equal(got["first_start_s"], np.array([r.first_start for r in want.reqs]))
+    assert np.array_equal(got["finish_s"], np.array([r.finished_at for r in want.reqs]))
+    assert np.array_equal(got["evictions"], np.array([r.evictions for r in want.reqs]))
+
+
+# ------------------------------------------------------------------------------- the hand-worked trace
+
+def golden_rows():
+    rows = []
+    for line in open(GOLDEN):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        t, kind, a, c = [x.strip() for x in line.split("|")]
+        rows.append((float(t), KINDS[kind], int(a), int(c)))
+    return rows
+
+
+def golden_inputs():
+    kw = dict(slots_interactive=1, slots_batch=2, rate_interactive=10.0, rate_batch=5.0, startup_s=4.0, tick_s=10.0,
+              theta=0.5, delta=0.1, floor_instances=2, initial_instances=2, max_batch_instances=4, groups_k=1,
+              z=0.0, mu_o_prior=100.0, sigma_o_prior=0.0, policy=0, horizon_s=0.0)
+    arrival = [0.0, 1.0, 2.0, 8.0, 8.0, 9.0, 105.0]
+    kind = [1, 0, 0, 1, 1, 1, 0]
+    tokens = [50.0, 30.0, 20.0, 400.0, 400.0, 400.0, 10.0]
+    slo = [100.0, 10.0, 10.0, 30.0, 30.0, 30.0, 10.0]
+    return kw, (arrival, kind, tokens, slo)
+
+
+def test_hand_worked_trace_oracle():
+    kw, trace = golden_inputs()
+    sim = ref.simulate(ref.SimConfig(**kw), *trace)
+    assert sim.log == golden_rows()
+    s = sim.summary()
+    assert s["evictions"] == 1 and s["instances_added"] == [0, 0, 1] and s["instances_removed"] == [0, 0, 1]
+    assert s["instance_seconds"][2] == pytest.approx(90.0)
+    assert s["batch_ttft_met"] == 4 and s["interactive_ttft_met"] == 3 and s["finished"] == 7
+
+
+def test_hand_worked_trace_library(b):
+    kw, trace = golden_inputs()
+    got = b.global_simulate(b.SimConfig(**kw), *trace, log_cap=1000)
+    assert got["log"] == golden_rows()
+    assert got["summary"]["evictions"] == 1 and got["summary"]["instances_added"] == [0, 0, 1]
+    assert got["summary"]["instance_seconds"][2] == pytest.approx(90.0)
+    assert list(got["first_start_s"]) == [0.0, 1.0, 2.0, 8.0, 14.0, 14.0, 105.0]
+    assert list(got["finish_s"]) == [7.0, 4.0, 4.0, 48.0, 94.0, 94.0, 106.0]
+    assert list(got["evictions"]) == [1, 0, 0, 0, 0, 0, 0]
+
+
+# ------------------------------------------------------------------------------- event-for-event parity
+
+@pytest.mark.parametrize("seed,cv,rate,frac,policy,over", [
+    (1, 1.0, 4.0, 0.3, 0, {}),                                            # Poisson arrivals, the paper's default
+    (2, 2.0, 4.0, 0.3, 0, {}),                                            # bursty
+    (3, 8.0, 3.0, 0.3, 0, {}),                                            # the paper's largest burstiness
+    (4, 1.0, 6.0, 0.6, 0, dict(slots_interactive=2, initial_instances=6)),  # few slots: many evictions
+    (5, 4.0, 5.0, 0.5, 1, {}),                                            # the immediate policy
+    (6, 1.0, 2.0, 1.0, 0, dict(groups_k=5)),                              # batch requests only
+    (7, 1.0, 2.0, 0.0, 0, {}),                                            # interactive requests only
+    (8, 1.0, 5.0, 0.4, 0, dict(startup_s=0.0, tick_s=1.0, delta=0.0)),    # instant start-up, no band
+    (9, 1.0, 8.0, 0.5, 0, dict(max_batch_instances=1, horizon_s=400.0)),  # capped and cut off
+])
+def test_event_for_event_against_the_oracle(b, seed, cv, rate, frac, policy, over):
+    n = 700
+    arrival, kind, tokens, slo = wl.request_trace(n, rate, cv, frac, seed, batch_ttft_s=300.0)
+    # a second class of batch requests with a short deadline, so that groups differ
+    slo = np.where((kind == 1) & (np.arange(n) % 3 == 0), 60.0, slo)
+    kw = base_config(policy=policy, **over)
+    got, want = run_both(b, kw, (arrival, kind, tokens, slo))
+    assert_same_run(got, want)
+    if not over.get("horizon_s"):
+        assert got["summary"]["finished"] == n
+
+
+# ------------------------------------------------------------------------------- invariants of any run
+
+def replay(log, kw, trace, n_initial):
+    """Walk the event log and check the physical constraints of the model."""
+    arrival, kind, tokens, slo = trace
+    ready, cls, load, where = set(range(n_initial)), {}, {}, {}
+    want_int = max(1, int(np.floor(kw["theta"] * n_initial + 0.5)))
+    for i in range(n_initial):
+        cls[i] = 0 if i < want_int else 1
+        load[i] = 0
+    last_t = 0.0
+    for t, ev, a, c in log:
+        assert t >= last_t
+        last_t = t
+        if ev == KINDS["ADD"]:
+            cls[a], load[a] = c, 0
+        elif ev == KINDS["READY"]:
+            ready.add(a)
+        elif ev == KINDS["REMOVE"]:
+            assert load[a] == 0, "an instance was removed with requests on it"
+            ready.discard(a); cls[a] = None
+        elif ev == KINDS["START"]:
+            assert c in ready and cls[c] is not None and a not in where
+            assert t >= arrival[a]
+            if kind[a] == 0:
+                assert cls[c] in (0, 1), "interactive request on a batch instance"
+            else:
+                assert cls[c] in (1, 2), "batch request on an interactive instance"
+            load[c] += 1
+            assert load[c] <= (kw["slots_batch"] if cls[c] == 2 else kw["slots_interactive"])
+            where[a] = c
+        elif ev in (KINDS["EVICT"], KINDS["FINISH"]):
+            assert where.pop(a) == c
+            load[c] -= 1
+            if ev == KINDS["EVICT"]:
+                assert kind[a] == 1 and cls[c] == 1, "only batch requests on mixed instances are evicted"
+
+
+def test_runs_respect_slots_classes_and_readiness(b):
+    for seed, policy in ((11, 0), (12, 1)):
+        kw = base_config(policy=policy, slots_interactive=3)
+        trace = wl.request_trace(900, 6.0, 2.0, 0.5, seed, batch_ttft_s=200.0)
+        got = b.global_simulate(b.SimConfig(**kw), *trace, log_cap=2_000_000)
+        replay(got["log"], kw, trace, kw["initial_instances"])
+        s = got["summary"]
+        assert s["finished"] == 900 and s["tokens_served"] == pytest.approx(float(trace[2].sum()))
+        served = got["finish_s"] - got["first_start_s"]
+        assert np.all(got["first_start_s"] >= trace[0])
+        assert np.all(served >= trace[2] / kw["rate_interactive"] - 1e-9)      # nobody is faster than the fastest rate
+
+
+# ------------------------------------------------------------------------------- what the paper says it does
+
+def spike_trace(base_rate, factor, seed, t_spike=300.0, spike_len=120.0, t_end=600.0):
+    """Interactive Poisson arrivals at base_rate, multiplied by `factor` during the spike window."""
+    rng = np.random.default_rng([seed, 0x5B1])
+    out, t = [], 0.0
+    while t < t_end:
+        rate = base_rate * (factor if t_spike <= t < t_spike + spike_len else 1.0)
+        t += rng.exponential(1.0 / rate)
+        out.append(t)
+    arrival = np.array(out)
+    n = arrival.size
+    return arrival, np.zeros(n, np.int32), wl.output_lengths(n, seed, median=150.0, sigma=0.5), np.full(n, 10.0)
+
+
+def test_theta_one_third_absorbs_a_threefold_spike(b):
+    """Section 5.2: with a tail spike of three times the mean rate, Theta = 1/3.  Instances take 60 s
+    to start (Section 2.3), so the spike must be carried by what is already there."""
+    # 2.4 requests/s of ~170 tokens at 20 tokens/s: ~20 running, 16 slots per instance
+    kw = base_config(slots_interactive=16, startup_s=60.0, initial_instances=6, floor_instances=3, delta=0.1)
+    got = b.global_simulate(b.SimConfig(**kw), *spike_trace(2.4, 3.0, 21))
+    s = got["summary"]
+    assert s["interactive_ttft_met"] == s["interactive_total"], "a 3x spike must not cost an interactive SLO at Theta = 1/3"
+    # the same pool under an eightfold spike does miss: the over-provisioning is what carried the first one
+    got8 = b.global_simulate(b.SimConfig(**kw), *spike_trace(2.4, 8.0, 21))
+    s8 = got8["summary"]
+    assert s8["interactive_ttft_met"] < s8["interactive_total"]
+
+
+def batch_heavy_trace(seed):
+    arrival, kind, tokens, slo = wl.request_trace(1500, 5.0, 1.0, 0.7, seed, batch_ttft_s=600.0)
+    return arrival, kind, tokens, slo
+
+
+def test_queueing_cuts_scaling_actions_compared_with_immediate_scaling(b):
+    """Section 2.3 ('Immediate autoscaling can lead to hysteresis'): adding an instance as soon as a
+    request does not fit and removing it as soon as it idles takes a multiple of the scaling actions
+    that deadline-driven scaling on the queued groups takes -- direction only, no factor is pinned."""
+    trace = batch_heavy_trace(31)
+    kw = base_config(slots_batch=8, startup_s=20.0)
+    chiron = b.global_simulate(b.SimConfig(**kw), *trace)["summary"]
+    immediate = b.global_simulate(b.SimConfig(**dict(kw, policy=1)), *trace)["summary"]
+    acts = lambda s: s["instances_added"][2] + s["instances_removed"][2]
+    assert chiron["batch_ttft_met"] == chiron["batch_total"]
+    assert acts(immediate) >= 3 * max(1, acts(chiron)), (acts(immediate), acts(chiron))
+    assert chiron["instance_seconds"][2] < immediate["instance_seconds"][2]     # and it costs less
+
+
+def test_no_backpressure_adds_no_batch_instance(b):
+    """A light batch load fits the spare capacity of the mixed instances: BBP stays 0 and Algorithm 2
+    never dispatches an instance."""
+    trace = wl.request_trace(600, 1.5, 1.0, 0.2, 41, batch_ttft_s=3600.0)
+    kw = base_config(slots_interactive=16, initial_instances=6, floor_instances=6)
+    s = b.global_simulate(b.SimConfig(**kw), *trace)["summary"]
+    assert s["instances_added"][2] == 0 and s["peak_instances"][2] == 0
+    assert s["batch_ttft_met"] == s["batch_total"] and s["finished"] == 600
+
+
+def test_batch_instances_retire_when_nothing_is_queued_or_served(b):
+    """Algorithm 2's last step: a burst of batch requests brings instances up; once the queue is empty
+    and nothing runs on them, all of them are removed."""
+    n = 400
+    arrival = np.concatenate([np.linspace(0.0, 1.0, n - 1), [4000.0]])       # a burst, then one straggler much later
+    kind = np.concatenate([np.ones(n - 1, np.int32), [0]])
+    tokens = wl.output_lengths(n, 51)
+    slo = np.where(kind == 1, 120.0, 10.0)
+    kw = base_config(initial_instances=2, floor_instances=2)
+    got = b.global_simulate(b.SimConfig(**kw), arrival, kind, tokens, slo, log_cap=100000)
+    s = got["summary"]
+    assert s["peak_instances"][2] >= 2
+    assert s["instances_added"][2] == s["instances_removed"][2]
+    removes = [t for t, ev, a, c in got["log"] if ev == KINDS["REMOVE"] and c == 2]
+    last_batch_finish = max(got["finish_s"][:n - 1])
+    assert removes and min(removes) >= last_batch_finish and max(removes) <= last_batch_finish + kw["tick_s"] + 1e-9
+
+
+def test_without_batch_requests_no_batch_instance_exists(b):
+    trace = wl.request_trace(500, 4.0, 2.0, 0.0, 61)
+    s = b.global_simulate(b.SimConfig(**base_config()), *trace)["summary"]
+    assert s["peak_instances"][2] == 0 and s["evictions"] == 0 and s["batch_total"] == 0
+
+
+def test_bad_inputs_are_rejected(b):
+    ok = ([0.0, 1.0], [0, 1], [10.0, 10.0], [10.0, 100.0])
+    with pytest.raises(b.CkvError):
+        b.global_simulate(b.SimConfig(**base_config(tick_s=0.0)), *ok)
+    with pytest.raises(b.CkvError):
+        b.global_simulate(b.SimConfig(**base_config()), [1.0, 0.5], *ok[1:])      # arrivals out of order
+    with pytest.raises(b.CkvError):
+        b.global_simulate(b.SimConfig(**base_config()), ok[0], [0, 2], *ok[2:])   # unknown kind
+    with pytest.raises(b.CkvError):
+        b.global_simulate(b.SimConfig(**base_config(policy=7)), *ok)

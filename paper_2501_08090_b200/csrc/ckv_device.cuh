@@ -540,9 +540,10 @@ struct AttnParams {
 // reference the exponentials were taken against (log2 domain), l[8] their sums, O[8][D] the
 // weighted value sums, one row per column.  In memory it is `rows` (ncp rows of D floats at some
 // pitch) plus 16 floats (m[8], l[8]).  ncp is the live column count rounded up to a power of two
-// (at least 128 / D), so that the ncp * D floats of the rows split evenly over the 32 lanes: lane
-// owns 4 * J consecutive floats of ONE row g (J = ncp * D / 128 float4 pieces starting at
-// element d0).  A lane therefore needs one factor per partial, not eight, and the code below has
+// (at least 128 / D), so that the ncp * D floats of the rows split evenly over the 32 lanes: the
+// 32 / ncp lanes of ONE row g take its float4 pieces in turn (lane r of the row owns pieces r,
+// r + 32 / ncp, ...: J = ncp * D / 128 of them), which keeps shared-memory reads conflict-free
+// and global stores coalesced.  A lane therefore needs one factor per partial, not eight, and the code below has
 // no per-column unrolling: it is small, which matters because every warp runs it once, after its
 // span, from an instruction cache that has held nothing but the streaming loop.
 //
@@ -552,7 +553,9 @@ struct AttnParams {
 // rows or stored as one partial again.  The order of summation depends only on t, never on which
 // warp does the work, so results are bit-identical from run to run.
 struct FoldGeom {
-    int ncp, J, g, d0;
+    int ncp, J, g;
+    int d0;                         // first element of the lane's first float4 piece
+    int dq;                         // elements between its consecutive pieces
 };
 
 __device__ __forceinline__ FoldGeom fold_geometry(int ncols, int D, int lane)
@@ -562,8 +565,10 @@ __device__ __forceinline__ FoldGeom fold_geometry(int ncols, int D, int lane)
     while (ncp < ncols) ncp *= 2;
     fg.ncp = ncp;
     fg.J = ncp * D / 128;
-    fg.g = lane * ncp / 32;
-    fg.d0 = (lane * 4 * fg.J) % D;
+    const int lanes_per_row = 32 / ncp;
+    fg.g = lane / lanes_per_row;
+    fg.d0 = (lane % lanes_per_row) * 4;
+    fg.dq = lanes_per_row * 4;
     return fg;
 }
 
@@ -602,7 +607,8 @@ struct FoldCtx {
     float *part_acc;                // [slots][8][D]
     float *part_ml;                 // [slots][16]
     uint32_t *status;
-    int ncols, G, qi_stride, lane;
+    int ncols, lane;
+    int out_off;                    // elements from a pair's first output row to this lane's first float4 piece
     FoldGeom fg;
 };
 
@@ -615,7 +621,7 @@ __device__ __forceinline__ float ld_shared_f32(uint32_t addr)
 
 // Start the bulk copies of one round (partials t0 .. t0 + cnt - 1) of a job with global sources.
 template <int D>
-__device__ __noinline__ void fold_fetch(const FoldJob j, const FoldCtx c, int t0)
+__device__ __forceinline__ void fold_fetch(const FoldJob j, const FoldCtx c, int t0)
 {
     const int cnt = min(j.cap, j.n - t0);
     const int row_bytes = c.fg.ncp * D * 4;
@@ -634,9 +640,9 @@ __device__ __noinline__ void fold_fetch(const FoldJob j, const FoldCtx c, int t0
 // their way (fold_fetch).  Returns the number of phases the job's mbarrier has completed, or -1 if
 // a bounded wait gave up (nothing is stored then).
 template <int D>
-__device__ __noinline__ int fold_finish(const FoldJob j, const FoldCtx c)
+__device__ __forceinline__ int fold_finish(const FoldJob j, const FoldCtx c)
 {
-    const int g = c.fg.g, d0 = c.fg.d0, J = c.fg.J;
+    const int g = c.fg.g, d0 = c.fg.d0, dq = c.fg.dq, J = c.fg.J;
     float M = -INFINITY, L = 0.f;
     float4 acc[8];
 #pragma unroll
@@ -657,7 +663,7 @@ __device__ __noinline__ int fold_finish(const FoldJob j, const FoldCtx c)
             if (!ok) return -1;
         }
         float Mr = -INFINITY;
-#pragma unroll 1
+#pragma unroll 2
         for (int i = 0; i < cnt; ++i) {
             const uint32_t ml = (t0 + i == j.alt_t) ? j.alt_base + j.alt_ml_off : j.base + i * j.stride + j.ml_off;
             Mr = fmaxf(Mr, ld_shared_f32(ml + 4 * g));
@@ -666,12 +672,14 @@ __device__ __noinline__ int fold_finish(const FoldJob j, const FoldCtx c)
         // exponentials are then taken against 0 and come out 0
         const float Mn = fmaxf(M, Mr);
         const float ref = Mn == -INFINITY ? 0.f : Mn;
-        const float sc = fast_exp2(M - ref);
-        M = Mn;
-        L *= sc;
+        if (t0 > 0) {                            // later rounds: bring what has been summed to the new reference
+            const float sc = fast_exp2(M - ref);
+            L *= sc;
 #pragma unroll
-        for (int q = 0; q < 8; ++q) { acc[q].x *= sc; acc[q].y *= sc; acc[q].z *= sc; acc[q].w *= sc; }
-#pragma unroll 1
+            for (int q = 0; q < 8; ++q) { acc[q].x *= sc; acc[q].y *= sc; acc[q].z *= sc; acc[q].w *= sc; }
+        }
+        M = Mn;
+#pragma unroll 2
         for (int i = 0; i < cnt; ++i) {
             const bool alt = t0 + i == j.alt_t;
             const uint32_t pb = alt ? j.alt_base : j.base + i * j.stride;
@@ -682,7 +690,7 @@ __device__ __noinline__ int fold_finish(const FoldJob j, const FoldCtx c)
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
                 if (q < J) {
-                    const float4 a = ld_shared_f32x4(rows + q * 16);
+                    const float4 a = ld_shared_f32x4(rows + q * dq * 4);
                     acc[q].x += f * a.x; acc[q].y += f * a.y; acc[q].z += f * a.z; acc[q].w += f * a.w;
                 }
             }
@@ -691,15 +699,15 @@ __device__ __noinline__ int fold_finish(const FoldJob j, const FoldCtx c)
     }
     if (j.out_rows != nullptr) {
         if (g < c.ncols) {
-            const float inv = 1.f / L;
-            uint16_t *row = j.out_rows + (size_t)(g / c.G) * c.qi_stride + (size_t)(g % c.G) * D + d0;
+            const float inv = __frcp_rn(L);
+            uint16_t *row = j.out_rows + c.out_off;
 #pragma unroll
             for (int q = 0; q < 8; ++q) {
                 if (q < J) {
                     uint2 packed;
                     packed.x = pack_bf16x2(acc[q].x * inv, acc[q].y * inv);
                     packed.y = pack_bf16x2(acc[q].z * inv, acc[q].w * inv);
-                    *(uint2 *)(row + q * 4) = packed;
+                    *(uint2 *)(row + q * dq) = packed;
                 }
             }
         }
@@ -707,7 +715,7 @@ __device__ __noinline__ int fold_finish(const FoldJob j, const FoldCtx c)
         float *rows = c.part_acc + (size_t)j.dst_slot * kMaxGroup * D + g * D + d0;
 #pragma unroll
         for (int q = 0; q < 8; ++q)
-            if (q < J) *(float4 *)(rows + q * 4) = acc[q];
+            if (q < J) *(float4 *)(rows + q * dq) = acc[q];
         if (d0 == 0) {
             c.part_ml[j.dst_slot * 2 * kMaxGroup + g] = M;
             c.part_ml[j.dst_slot * 2 * kMaxGroup + kMaxGroup + g] = L;
@@ -717,7 +725,7 @@ __device__ __noinline__ int fold_finish(const FoldJob j, const FoldCtx c)
 #pragma unroll
             for (int q = 0; q < 8; ++q)
                 if (q < J)
-                    asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(crow + q * 16), "f"(acc[q].x), "f"(acc[q].y),
+                    asm volatile("st.shared.v4.f32 [%0], {%1,%2,%3,%4};" ::"r"(crow + q * dq * 4), "f"(acc[q].x), "f"(acc[q].y),
                                  "f"(acc[q].z), "f"(acc[q].w) : "memory");
             if (d0 == 0) {
                 asm volatile("st.shared.f32 [%0], %1;" ::"r"(j.copy_base + j.copy_ml_off + 4 * g), "f"(M) : "memory");
@@ -1245,8 +1253,9 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     // with its own; a pair cut into more than kTreeFrom partials is folded in two levels.
     FoldCtx fc;
     fc.part_acc = p.part_acc; fc.part_ml = p.part_ml; fc.status = p.status;
-    fc.ncols = ncols; fc.G = G; fc.qi_stride = qi_stride; fc.lane = lane;
+    fc.ncols = ncols; fc.lane = lane;
     fc.fg = fold_geometry(ncols, D, lane);
+    fc.out_off = (fc.fg.g / G) * qi_stride + (fc.fg.g % G) * D + fc.fg.d0;
     const uint32_t staging_u32 = smem_u32(smem + Lay::kStagingOff), park_u32 = smem_u32(smem + Lay::kParkOff);
     constexpr int kStagingMl = kMaxGroup * Lay::kStagePitch * 4, kParkMl = kMaxGroup * D * 4;
     const int part_bytes = fc.fg.ncp * D * 4 + 64;               // a fetched partial in the ring: rows, then (m, l)

@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on the headline
 # workload, from the ncu capture summarised in profiles/paged_decode_attn_llama8b_b64.md.  Set to
 # None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES = 573.8e6    # dram read + write per launch of the attention kernel, mean of 2 captured launches
+NCU_TRAFFIC_BYTES = None       # dram read + write per launch of the attention kernel (ncu); None: not captured for this kernel
 
 
 # ------------------------------------------------------------------------------- clocks
@@ -272,6 +272,38 @@ def cpu_baseline(name: str, target_s: float = 12.0) -> dict:
             "us_per_step_sample": t * 1e6}
 
 
+def oracle_beside(name: str, batch=None, max_tokens: int = 250_000, passes: int = 2) -> dict:
+    """The oracle timed on a bounded sample of another workload: the first requests of the batch whose
+    contexts add up to at most max_tokens (one layer), extrapolated to the whole step by algorithmic bytes."""
+    from oracle import oracle
+    from oracle.oracle import PoolShape
+    w = wl.workload(name)
+    lens_all = wl.seq_lens(w, batch)
+    take = max(1, int(np.searchsorted(np.cumsum(lens_all.astype(np.int64)), max_tokens, side="right")))
+    lens = lens_all[:take]
+    if int(lens.sum()) > 4 * max_tokens:              # a single very long request: time a prefix of it
+        lens = np.minimum(lens, max_tokens).astype(np.int32)
+    npg = int(wl.pages_of(lens).sum())
+    bt = wl.block_tables(lens, npg, w.seed)
+    sh = PoolShape(1, npg, w.num_q_heads, w.num_kv_heads, w.page_size, w.head_dim)
+    pool = wl.normal_bf16((wl.pool_elems(w, npg, 1),), w.seed, 11)
+    q = wl.normal_bf16((lens.size, w.num_q_heads, w.head_dim), w.seed, 12)
+    k = wl.normal_bf16((lens.size, w.num_kv_heads, w.head_dim), w.seed, 13)
+    times = []
+    for _ in range(passes + 1):
+        t0 = time.perf_counter()
+        assert oracle.kv_append(pool, sh, 0, bt, lens, k, k) == 0
+        oracle.decode_attention(pool, sh, 0, bt, lens, q)
+        times.append(time.perf_counter() - t0)
+    t = min(times[1:])                                 # the first pass pays for page faults
+    sample_bytes = wl.algorithmic_bytes(w, lens, 1)["total"]
+    full_bytes = wl.algorithmic_bytes(w, lens_all)["total"]
+    return {"value": sample_bytes / t / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": "%d of %d requests (%d of %d tokens), 1 of %d layers; best of %d passes"
+                      % (lens.size, lens_all.size, int(lens.sum()), int(lens_all.sum()), w.num_layers, passes),
+            "us_per_step_extrapolated": t * 1e6 * full_bytes / sample_bytes}
+
+
 def run_reference(args) -> None:
     """--impl reference: K timed oracle steps on a sample sized so the run ends within minutes."""
     rank = int(os.environ.get("RANK", "0"))
@@ -379,10 +411,13 @@ def run_ours(args) -> None:
     h2d = sum(hb[k].numel() * hb[k].element_size() for k in hb)
     d2h = hout.numel() * hout.element_size()
 
+    host_calls = [dw.kp.host_step_call(layer, hb["bt"], hb["sl"], hb["q"], hb["k"], hb["v"], hout)
+                  for layer in range(w.num_layers)]
+
     def e2e_steps(n):
         for _ in range(n):
-            for layer in range(w.num_layers):
-                dw.kp.decode_step_host(layer, hb["bt"], hb["sl"], hb["q"], hb["k"], hb["v"], hout)
+            for call in host_calls:
+                call()
     e2e_steps(3)
     barrier(world)
     t0 = time.perf_counter()
@@ -391,7 +426,9 @@ def run_ours(args) -> None:
     e2e_s = time.perf_counter() - t0
     e2e_ms_max, e2e_bytes = reduce_max_sum(e2e_s * 1e3, float(dw.bytes["total"]) * E, world)
     e2e = {"value": e2e_bytes / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d * w.num_layers,
-           "d2h_bytes_per_step": d2h * w.num_layers, "steps": E, "us_per_step": e2e_ms_max / E * 1e3}
+           "d2h_bytes_per_step": d2h * w.num_layers, "steps": E, "us_per_step": e2e_ms_max / E * 1e3,
+           "route": "decode_step_host, pinned host buffers: gather kernel in, output rows written to host memory by the "
+                    "attention kernel, one synchronise per step"}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
@@ -404,6 +441,9 @@ def run_ours(args) -> None:
                    "instances": "one independent batch per GPU"},
         "us_per_step": ms_max / K * 1e3, "tokens_per_s": tokens_all / (ms_max * 1e-3),
         "kv_gbs": kv_all / (ms_max * 1e-3) / 1e9, "frac_of_8TBs": value / NORMALISED_TO_TBS,
+        # the same launch standing alone (events around every launch: what an engine that runs other
+        # kernels between attention launches sees)
+        "isolated_us_per_launch": attn_ms / attn_n * 1e3, "isolated_frac_of_8TBs": isolated / (NORMALISED_TO_TBS * 1e3),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches_all), "roofline": roofline,
     }
 
@@ -412,6 +452,7 @@ def run_ours(args) -> None:
             line["latency_sweep"] = run_sweep(dev)
             line["local_autoscaler"] = run_autoscaler(line["latency_sweep"])
             line["global_autoscaler"] = run_global_autoscaler(line["local_autoscaler"])
+            line["global_autoscaler"]["simulation"] = run_global_simulation(line["local_autoscaler"])
             line["kv_swap"] = run_swap(dev)
             line["multi_token_step"] = run_multi_token(dw)
             dw.kp.close()
@@ -421,6 +462,7 @@ def run_ours(args) -> None:
             line["cuda_graph"] = run_cuda_graph(dev)
         if not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(HEADLINE)
+            add_oracle_timings(line)
     if name != HEADLINE:
         line["roofline"]["traffic"] = None            # the ncu figure belongs to the headline workload
     if rank == 0:
@@ -446,6 +488,16 @@ def run_sweep(dev) -> dict:
                      "tokens_per_s": round(b / (m * 1e-6)), "tbs": round(nb / (m * 1e-6) / 1e12, 3)})
     dw.kp.close()
     return {"workload": "mixed_sweep", "l2": "before every timed step 256 MB are overwritten, then another 256 MB read (cold and clean L2)", "points": rows}
+
+
+def add_oracle_timings(line: dict) -> None:
+    """The oracle timed beside the other workloads of the line (rank 0, after the GPU work is done)."""
+    for row in line.get("latency_sweep", {}).get("points", []):
+        if row["batch"] in (1, 64, 512):
+            row["cpu_baseline"] = oracle_beside("mixed_sweep", batch=row["batch"])
+    for row in line.get("other_workloads", []):
+        if "skipped" not in row:
+            row["cpu_baseline"] = oracle_beside(row["workload"])
 
 
 def run_swap(dev) -> dict:
@@ -619,6 +671,37 @@ def run_global_autoscaler(local: dict) -> dict:
     for busy in (3, 5, 8, 4, 1):
         total = binding.interactive_autoscale(busy, total, 1.0 / 3.0, 0.05)
         out["interactive"].append({"busy": busy, "instances": total})
+    return out
+
+
+def run_global_simulation(local: dict) -> dict:
+    """Sections 3 and 5 in time: a seeded Poisson trace of interactive and batch requests (Section 6
+    "Workloads": TTFT SLOs of 10 s and one hour, here 10 s and 10 minutes to keep the run short) served by
+    instances whose batch sizes and per-request token rates are what Algorithm 1 settled at on the measured
+    latency curve; the deadline-driven policy beside immediate scaling (Section 2.3)."""
+    from paper_2501_08090_b200 import binding
+    inter, batch = local["runs"][0], local["runs"][-1]
+    kw = dict(slots_interactive=max(1, inter["trough_batch"]), slots_batch=max(1, batch["trough_batch"]),
+              rate_interactive=1e3 / inter["max_itl_ms"], rate_batch=1e3 / batch["max_itl_ms"],
+              startup_s=30.0, tick_s=5.0, theta=1.0 / 3.0, delta=0.05, floor_instances=1, initial_instances=3,
+              max_batch_instances=64, groups_k=4, z=2.33, mu_o_prior=200.0, sigma_o_prior=150.0, policy=0, horizon_s=0.0)
+    # arrival rate that keeps about three interactive instances busy
+    mean_tokens = float(wl.output_lengths(4000, 7).mean())
+    rate = 0.9 * 3 * kw["slots_interactive"] * kw["rate_interactive"] / mean_tokens / 0.5
+    trace = wl.request_trace(4000, rate, 1.0, 0.5, seed=7, batch_ttft_s=600.0)
+    out = {"instance_model": {k: (round(v, 3) if isinstance(v, float) else v) for k, v in kw.items() if k.startswith(("slots", "rate"))},
+           "requests": 4000, "arrival_rate_per_s": round(rate, 2), "policies": []}
+    for policy, name in ((0, "deadline-driven (Algorithm 2 on request groups)"), (1, "immediate")):
+        t0 = time.perf_counter()
+        r = binding.global_simulate(binding.SimConfig(**dict(kw, policy=policy)), *trace)
+        s = r["summary"]
+        out["policies"].append({"policy": name, "events": r["events"], "wall_ms": round((time.perf_counter() - t0) * 1e3, 1),
+                                "interactive_ttft_met": s["interactive_ttft_met"] / max(1, s["interactive_total"]),
+                                "batch_ttft_met": s["batch_ttft_met"] / max(1, s["batch_total"]),
+                                "instance_hours": [round(x / 3600.0, 3) for x in s["instance_seconds"]],
+                                "scale_ups": s["instances_added"], "scale_downs": s["instances_removed"],
+                                "hysteresis": round((sum(s["instances_added"]) + sum(s["instances_removed"])) / max(1, sum(s["instances_added"])), 2),
+                                "evictions": s["evictions"], "end_s": round(s["end_s"], 1)})
     return out
 
 

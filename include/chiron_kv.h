@@ -221,14 +221,40 @@ int32_t ckv_set_overlap(ckv_pool *pool, int32_t enable);
 int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits);
 
 /*
+ * Self-test of the failure path behind CKV_ETIMEOUT (test support; not part of the decode path).
+ * Every wait inside the kernels is bounded: a warp that waits longer than the limit for a copy to
+ * land sets CKV_STATUS_WAIT_LIMIT, stops working and returns, so a lost copy becomes an error
+ * code instead of a hung GPU.  This call makes that happen on purpose and harmlessly: it enqueues
+ * a one-warp kernel that waits, with the kernels' own wait routine and `limit_ns` as the limit
+ * (1 us .. 100 ms), on a barrier phase that nothing completes -- no copy is issued -- and that
+ * leaves arrival counter 0 raised by one, as a warp giving up inside a merge would.  Afterwards
+ * kv_check_status() must report CKV_ETIMEOUT and bring the handle back to a usable state (status
+ * word and arrival counters cleared).  Errors: CKV_EINVAL, CKV_ECUDA.
+ */
+int32_t ckv_wait_limit_selftest(ckv_pool *pool, uint64_t limit_ns, void *stream);
+
+/*
  * One whole iteration for one layer with HOST buffers: brings the tables, lengths, q, k_new and
  * v_new to the device, runs decode_step, delivers the output to h_out and synchronises `stream`.
- * If the device can address all six buffers (pinned or registered host memory, h_out 16-byte
- * aligned) nothing is copied by DMA: one kernel gathers the five inputs into the workspace and
- * the attention kernel writes its output rows straight into h_out (two launches); otherwise five
- * host-to-device copies, decode_step and one device-to-host copy are issued.
+ * Routes (ckv_set_host_route; CKV_HOST_ROUTE_AUTO picks STAGED when it applies, else COPY):
+ *   CKV_HOST_ROUTE_STAGED  all six buffers are host memory the device can address (pinned or
+ *                          registered, h_out 16-byte aligned): one kernel gathers the five inputs
+ *                          into the workspace, the attention kernel starts under it, waits for it
+ *                          before its plan and writes its output rows straight into h_out.  Two
+ *                          launches, no DMA copy.
+ *   CKV_HOST_ROUTE_DIRECT  same buffers (q, k_new, v_new 16-byte aligned too): the attention kernel
+ *                          reads everything straight from host memory.  One launch; every read
+ *                          pays the host link's latency.
+ *   CKV_HOST_ROUTE_COPY    any host memory: five host-to-device copies, decode_step, one
+ *                          device-to-host copy.
+ * A route whose conditions are not met falls back to the next one in this order.
  * h_out: bf16 [batch][num_q_heads][head_dim].  Errors: as kv_append / decode_attention.
  */
+#define CKV_HOST_ROUTE_AUTO   0
+#define CKV_HOST_ROUTE_STAGED 1
+#define CKV_HOST_ROUTE_DIRECT 2
+#define CKV_HOST_ROUTE_COPY   3
+int32_t ckv_set_host_route(ckv_pool *pool, int32_t route);
 int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch,
                          const int32_t *h_block_tables, const int32_t *h_seq_lens,
                          const void *h_q, const void *h_k_new, const void *h_v_new,
@@ -236,8 +262,8 @@ int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch,
 
 /*
  * Iteration latency against batch size: the curve Algorithm 1 reads as ITL(batch size)
- * (Section 2.1, figure "Variation in inter-token latency and token throughput with
- * increasing batch size"; Section 4.1).  For each i < n_sizes, runs `warmup` untimed and `iters` timed
+ * (Section 2.1, the figure of ITL and throughput against batch size; Section 4.1).  For each
+ * i < n_sizes, runs `warmup` untimed and `iters` timed
  * steps on the first batch_sizes[i] requests of the given arrays; a step is decode_step (append
  * + attention in one kernel) for every layer.  Per-layer inputs are laid out
  *   d_q, d_out [num_layers][batch_stride][Hq][d],  d_k_new, d_v_new [num_layers][batch_stride][Hkv][d].
@@ -320,12 +346,17 @@ int32_t kv_swap_in(ckv_pool *pool, int32_t n_pages, const int32_t *d_page_ids, c
  *   d_pool     256-byte aligned device pointer to kv_pool_bytes(cfg) bytes
  *   num_spans  partition width; 0 = warps per CTA x number of SMs.  More than 640 is rejected
  *              with CKV_EINVAL and a message -- nothing is launched.
- *   h_status   NULL: the call only enqueues work on `stream`.  Otherwise the call synchronises
- *              `stream`, stores the CKV_STATUS_* bits there and returns CKV_EBOUNDS /
- *              CKV_ETIMEOUT if any is set.
+ *   h_status   NULL: the call only enqueues work on `stream`; the device status bits of this call
+ *              (bad length, bad page id, wait limit) can then not be read afterwards -- the next
+ *              call clears them -- so pass NULL only for inputs known to be valid.  Otherwise the
+ *              call synchronises `stream`, stores the CKV_STATUS_* bits there and returns
+ *              CKV_EBOUNDS / CKV_ETIMEOUT if any is set.
  *
  * Set-up: the first call on each device looks up the array's device address
- * (cudaGetSymbolAddress) and remembers it; make that first call outside any stream capture.
+ * (cudaGetSymbolAddress), the device's SM count and the kernel's shared-memory attribute and
+ * remembers them; make that first call outside any stream capture.  First calls from several
+ * host threads at once are harmless (every thread would store the same values).  Later calls do
+ * no look-ups: they encode the tensor map of the pool on the stack, clear the counters and launch.
  * Sharing: every call on a device uses the same array, which still holds the previous call's
  * contents; each call clears the parts that must start at zero (status word, arrival counters) on
  * `stream` before its kernel.  Two calls that can overlap on the GPU (different streams, no

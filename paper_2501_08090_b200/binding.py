@@ -18,6 +18,7 @@ LIBRARY = os.path.join(_HERE, "libchiron_kv.so")
 
 CKV_OK, CKV_EINVAL, CKV_ENOMEM, CKV_ECUDA, CKV_EBOUNDS, CKV_ETIMEOUT = 0, -1, -2, -3, -4, -5
 STATUS_BAD_LENGTH, STATUS_BAD_PAGE, STATUS_WAIT_LIMIT = 1, 2, 4
+HOST_ROUTE_AUTO, HOST_ROUTE_STAGED, HOST_ROUTE_DIRECT, HOST_ROUTE_COPY = 0, 1, 2, 3
 TILE_TOKENS, PIECE_COST_TILES = 32, 2      # the plan's tile size and per-piece overhead units
 
 EXPORTS = (
@@ -26,7 +27,7 @@ EXPORTS = (
     "decode_step_host", "step_latency_sweep", "ckv_profile_enable", "ckv_profile_read",
     "ckv_launch_count", "ckv_last_error", "ckv_read_span_trace", "ckv_set_overlap",
     "decode_attention_noalloc", "decode_step", "kv_swap_out", "kv_swap_in",
-    "kv_append_multi", "decode_attention_multi", "kv_read_probe",
+    "kv_append_multi", "decode_attention_multi", "kv_read_probe", "ckv_wait_limit_selftest", "ckv_set_host_route",
     "local_autoscaler_instance_slo", "local_autoscaler_create", "local_autoscaler_destroy",
     "local_autoscaler_update", "local_autoscaler_get", "local_autoscaler_simulate",
     "global_request_groups", "global_waiting_time", "global_batch_backpressure", "global_batch_autoscale",
@@ -95,10 +96,12 @@ def _load() -> ctypes.CDLL:
     lib.kv_append_multi.restype = i32; lib.kv_append_multi.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.decode_attention_multi.restype = i32; lib.decode_attention_multi.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.kv_read_probe.restype = i32; lib.kv_read_probe.argtypes = [vp, i32, i32, vp, vp, vp]
+    lib.ckv_wait_limit_selftest.restype = i32; lib.ckv_wait_limit_selftest.argtypes = [vp, ctypes.c_uint64, vp]
     lib.decode_plan.restype = i32; lib.decode_plan.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.ckv_set_partition.restype = i32; lib.ckv_set_partition.argtypes = [vp, i32]
     lib.ckv_set_overlap.restype = i32; lib.ckv_set_overlap.argtypes = [vp, i32]
     lib.ckv_get_partition.restype = i32; lib.ckv_get_partition.argtypes = [vp]
+    lib.ckv_set_host_route.restype = i32; lib.ckv_set_host_route.argtypes = [vp, i32]
     lib.kv_check_status.restype = i32; lib.kv_check_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.decode_step_host.restype = i32; lib.decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]
     lib.step_latency_sweep.restype = i32
@@ -273,6 +276,10 @@ class KvPool:
         _check(lib.kv_read_probe(self._h, layer, int(seq_lens.shape[0]), _dev_ptr(block_tables, torch.int32),
                                  _dev_ptr(seq_lens, torch.int32), _stream_ptr(stream)))
 
+    def wait_limit_selftest(self, limit_ns: int, stream=None) -> None:
+        """Make a bounded device-side wait run out on purpose (see ckv_wait_limit_selftest)."""
+        _check(lib.ckv_wait_limit_selftest(self._h, int(limit_ns), _stream_ptr(stream)))
+
     def decode_plan(self, seq_lens, stream=None):
         """(header dict, int32 [num_spans][4] array of span starts)."""
         batch = int(seq_lens.shape[0])
@@ -308,6 +315,27 @@ class KvPool:
         _check(lib.decode_step_host(self._h, layer, batch, block_tables.data_ptr(), seq_lens.data_ptr(),
                                     q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
                                     _stream_ptr(stream)))
+
+    def set_host_route(self, route: int) -> None:
+        """How decode_step_host moves its buffers: HOST_ROUTE_AUTO / STAGED / DIRECT / COPY."""
+        _check(lib.ckv_set_host_route(self._h, int(route)))
+
+    def host_step_call(self, layer: int, block_tables, seq_lens, q, k_new, v_new, out, stream=None):
+        """decode_step_host with its arguments marshalled once: returns a callable that issues one
+        step per call (for loops that reuse the same host buffers; the buffers must stay alive)."""
+        for t in (block_tables, seq_lens, q, k_new, v_new, out):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("decode_step_host takes contiguous host tensors")
+        keep = (block_tables, seq_lens, q, k_new, v_new, out)
+        args = (self._h, int(layer), int(seq_lens.shape[0]), block_tables.data_ptr(), seq_lens.data_ptr(),
+                q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(), _stream_ptr(stream))
+        fn = lib.decode_step_host
+
+        def call(_keep=keep):
+            rc = fn(*args)
+            if rc != CKV_OK:
+                raise CkvError(rc, last_error())
+        return call
 
     def step_latency_sweep(self, batch_sizes: Sequence[int], block_tables, seq_lens, q, k_new, v_new, out,
                            warmup: int = 3, iters: int = 20, flush: Optional[torch.Tensor] = None,

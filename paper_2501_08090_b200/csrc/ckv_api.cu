@@ -7,6 +7,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -111,6 +112,41 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
+// cuTensorMapEncodeTiled, looked up once per process (the driver library is not linked).
+EncodeTiledFn encode_tiled_fn(const char **why)
+{
+    static EncodeTiledFn cached = nullptr;
+    if (cached) return cached;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    const cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+        *why = cudaGetErrorString(e);
+        return nullptr;
+    }
+    cached = reinterpret_cast<EncodeTiledFn>(fn);
+    return cached;
+}
+
+// Tensor map over a whole pool seen as rows of head_dim bf16; one box = 32 rows (the 16 key rows
+// and 16 value rows of one (page, kv head)) x 64 columns, stored with the 128-byte swizzle.
+int32_t encode_pool_map(const ckv_config *cfg, const void *d_pool, CUtensorMap *out, const char *fn_name)
+{
+    const char *why = "";
+    const EncodeTiledFn encode = encode_tiled_fn(&why);
+    if (!encode) return fail(CKV_ECUDA, "%s: cuTensorMapEncodeTiled not available (%s)", fn_name, why);
+    const cuuint64_t rows = (cuuint64_t)cfg->num_layers * cfg->num_pages * cfg->num_kv_heads * 32;
+    const cuuint64_t dims[2] = {(cuuint64_t)cfg->head_dim, rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cfg->head_dim * 2};
+    const cuuint32_t box[2] = {64, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult cr = encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(d_pool), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (cr != CUDA_SUCCESS) return fail(CKV_ECUDA, "%s: cuTensorMapEncodeTiled returned %d", fn_name, (int)cr);
+    return CKV_OK;
+}
+
 }  // namespace
 
 struct ckv_pool {
@@ -126,6 +162,8 @@ struct ckv_pool {
     bool profile;
     bool overlap;                    // launch kernels with programmatic stream serialization
     bool pool_written;               // a kernel other than the fused step wrote the pool since the last attention launch
+    bool inputs_from_predecessor;    // the next attention launch reads tables and lengths its predecessor in the stream writes
+    int host_route;                  // decode_step_host: CKV_HOST_ROUTE_*
     std::vector<cudaEvent_t> ev;     // pairs (start, stop)
     int ev_used;
 
@@ -162,6 +200,9 @@ int32_t launch_attention(ckv_pool *pool, const ckv::AttnParams &ap, cudaStream_t
 int32_t check_call(ckv_pool *pool, int32_t layer, int32_t batch, const char *fn)
 {
     if (!pool) return fail(CKV_EINVAL, "%s: pool is NULL", fn);
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess || current != pool->device)
+        return fail(CKV_EINVAL, "%s: the pool lives on device %d but device %d is current", fn, pool->device, current);
     if (layer < 0 || layer >= pool->cfg.num_layers)
         return fail(CKV_EINVAL, "%s: layer %d outside [0, %d)", fn, layer, pool->cfg.num_layers);
     if (batch < 1 || batch > pool->cfg.max_batch)
@@ -215,7 +256,13 @@ int32_t launch_attention_noalloc(const CUtensorMap &tmap, const ckv::AttnParams 
 {
     using Lay = ckv::AttnLayout<D, W, NS>;
     auto kernel = ckv::paged_decode_attn_kernel<D, W, NS, false>;
-    CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
+    static bool configured[kMaxDevices] = {};                     // per device: the attribute is set once
+    int device = 0;
+    CKV_CUDA(cudaGetDevice(&device));
+    if (!configured[device]) {
+        CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
+        configured[device] = true;
+    }
     kernel<<<(ap.num_spans + W - 1) / W, Lay::kThreads, Lay::kSmemBytes, stream>>>(tmap, ap);
     CKV_CUDA(cudaGetLastError());
     return CKV_OK;
@@ -286,29 +333,13 @@ int32_t kv_pool_create(const ckv_config *cfg, void *d_pool, size_t pool_bytes, v
     p->profile = false;
     p->overlap = true;
     p->pool_written = false;
+    p->inputs_from_predecessor = false;
+    p->host_route = CKV_HOST_ROUTE_AUTO;
     p->ev_used = 0;
 
-    // Tensor map over the whole pool seen as rows of head_dim bf16; one box = 32 rows (the 16 key
-    // rows and 16 value rows of one (page, kv head)) x 64 columns, stored with the 128-byte swizzle.
-    void *fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+    if (int32_t rc = encode_pool_map(cfg, d_pool, &p->tmap, "kv_pool_create")) {
         delete p;
-        return fail(CKV_ECUDA, "kv_pool_create: cuTensorMapEncodeTiled not available (%s)", cudaGetErrorString(e));
-    }
-    const cuuint64_t rows = (cuuint64_t)cfg->num_layers * cfg->num_pages * cfg->num_kv_heads * 32;
-    const cuuint64_t dims[2] = {(cuuint64_t)cfg->head_dim, rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cfg->head_dim * 2};
-    const cuuint32_t box[2] = {64, 32};
-    const cuuint32_t estr[2] = {1, 1};
-    CUresult cr = reinterpret_cast<EncodeTiledFn>(fn)(&p->tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, d_pool, dims,
-                                                      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (cr != CUDA_SUCCESS) {
-        delete p;
-        return fail(CKV_ECUDA, "kv_pool_create: cuTensorMapEncodeTiled returned %d", (int)cr);
+        return rc;
     }
     cudaError_t me = cudaMemset(d_workspace, 0, ws.total);
     if (me == cudaSuccess) me = cudaDeviceSynchronize();
@@ -344,6 +375,14 @@ int32_t ckv_set_overlap(ckv_pool *pool, int32_t enable)
 {
     if (!pool) return fail(CKV_EINVAL, "ckv_set_overlap: pool is NULL");
     pool->overlap = enable != 0;
+    return CKV_OK;
+}
+
+int32_t ckv_set_host_route(ckv_pool *pool, int32_t route)
+{
+    if (!pool) return fail(CKV_EINVAL, "ckv_set_host_route: pool is NULL");
+    if (route < CKV_HOST_ROUTE_AUTO || route > CKV_HOST_ROUTE_COPY) return fail(CKV_EINVAL, "ckv_set_host_route: unknown route %d", route);
+    pool->host_route = route;
     return CKV_OK;
 }
 
@@ -446,8 +485,9 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
     ap.q_pass = q_len;
     // A fused step may start loading tiles under its predecessor's tail -- unless that predecessor
     // may be a kernel of this library that writes the pool (an append or a swap-in).
-    ap.early_loads = pool->pool_written ? 0 : 1;
+    ap.early_loads = pool->inputs_from_predecessor ? -1 : pool->pool_written ? 0 : 1;
     pool->pool_written = false;
+    pool->inputs_from_predecessor = false;
     ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)c.head_dim));
 
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -567,6 +607,18 @@ int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits)
     return CKV_OK;
 }
 
+int32_t ckv_wait_limit_selftest(ckv_pool *pool, uint64_t limit_ns, void *stream)
+{
+    if (!pool) return fail(CKV_EINVAL, "ckv_wait_limit_selftest: pool is NULL");
+    if (limit_ns < 1000 || limit_ns > 100000000ull)
+        return fail(CKV_EINVAL, "ckv_wait_limit_selftest: limit outside [1 us, 100 ms]");
+    ckv::wait_limit_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        pool->wsp<uint32_t>(pool->ws.status), pool->wsp<int32_t>(pool->ws.arrivals), limit_ns);
+    CKV_CUDA(cudaGetLastError());
+    pool->launches += 1;
+    return CKV_OK;
+}
+
 // Device-visible address of a host buffer if the device can address it (pinned or registered
 // memory), else NULL.
 static void *mapped_or_null(const void *h)
@@ -596,14 +648,25 @@ int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch, const int
     const size_t n_bt = sizeof(int32_t) * (size_t)batch * c.max_pages_per_req, n_sl = sizeof(int32_t) * (size_t)batch;
     const size_t n_q = (size_t)batch * c.num_q_heads * d2, n_kv = (size_t)batch * c.num_kv_heads * d2;
 
-    // Pinned buffers the device can address: one gather kernel brings all five inputs over, and
-    // the attention kernel writes its output rows straight into the host buffer -- two launches
-    // instead of six copies and one.  The tables and lengths come from the kernel just before, so
-    // this launch takes plain stream order.
+    // Pinned buffers the device can address take one of two routes without a DMA copy; both write
+    // the output rows straight into the host buffer.
+    //   staged: one gather kernel brings the five inputs into the workspace, the attention kernel
+    //           follows it with programmatic serialization and waits for it before its plan;
+    //   direct: the attention kernel reads tables, lengths, q and the new rows straight from host
+    //           memory (one launch; every read crosses the host link with its latency).
     const void *m_bt = mapped_or_null(h_block_tables), *m_sl = mapped_or_null(h_seq_lens), *m_q = mapped_or_null(h_q);
     const void *m_k = mapped_or_null(h_k_new), *m_v = mapped_or_null(h_v_new);
     void *m_o = mapped_or_null(h_out);
-    if (m_bt && m_sl && m_q && m_k && m_v && m_o && aligned16(m_o)) {
+    const bool all_mapped = m_bt && m_sl && m_q && m_k && m_v && m_o && aligned16(m_o);
+    const bool direct_ok = all_mapped && aligned16(m_q) && aligned16(m_k) && aligned16(m_v);
+    if (direct_ok && pool->host_route == CKV_HOST_ROUTE_DIRECT) {
+        const int32_t rc = decode_step(pool, layer, batch, static_cast<const int32_t *>(m_bt), static_cast<const int32_t *>(m_sl),
+                                       m_q, m_k, m_v, m_o, stream);
+        if (rc) return rc;
+        CKV_CUDA(cudaStreamSynchronize(s));
+        return CKV_OK;
+    }
+    if (all_mapped && pool->host_route != CKV_HOST_ROUTE_COPY) {
         ckv::GatherParams gp{};
         const void *src[5] = {m_bt, m_sl, m_q, m_k, m_v};
         void *dst[5] = {d_bt, d_sl, d_q, d_k, d_v};
@@ -619,10 +682,8 @@ int32_t decode_step_host(ckv_pool *pool, int32_t layer, int32_t batch, const int
         ckv::host_gather_kernel<<<blocks, 256, 0, s>>>(gp);
         CKV_CUDA(cudaGetLastError());
         pool->launches += 1;
-        const bool overlap = pool->overlap;
-        pool->overlap = false;
+        pool->inputs_from_predecessor = true;    // the attention kernel starts under the gather and waits for it first
         const int32_t rc = decode_step(pool, layer, batch, d_bt, d_sl, d_q, d_k, d_v, m_o, stream);
-        pool->overlap = overlap;
         if (rc) return rc;
         CKV_CUDA(cudaStreamSynchronize(s));
         return CKV_OK;
@@ -658,9 +719,20 @@ int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch
     const size_t q_layer = (size_t)batch_stride * c.num_q_heads * d2;
     const size_t kv_layer = (size_t)batch_stride * c.num_kv_heads * d2;
 
-    std::vector<cudaEvent_t> ev(2 * (size_t)iters);
-    for (auto &e : ev) CKV_CUDA(cudaEventCreate(&e));
+    std::vector<cudaEvent_t> ev(2 * (size_t)iters, nullptr);
     int32_t rc = CKV_OK;
+    for (auto &e : ev) {
+        const cudaError_t ce = cudaEventCreate(&e);
+        if (ce != cudaSuccess) {
+            e = nullptr;
+            rc = fail(CKV_ECUDA, "step_latency_sweep: cudaEventCreate failed: %s", cudaGetErrorString(ce));
+            break;
+        }
+    }
+    auto record = [&](cudaEvent_t e) {
+        const cudaError_t ce = cudaEventRecord(e, s);
+        if (ce != cudaSuccess && rc == CKV_OK) rc = fail(CKV_ECUDA, "step_latency_sweep: cudaEventRecord failed: %s", cudaGetErrorString(ce));
+    };
     std::vector<float> ms((size_t)iters);
     for (int i = 0; i < n_sizes && rc == CKV_OK; ++i) {
         const int32_t b = batch_sizes[i];
@@ -678,7 +750,7 @@ int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch
                 e = cudaGetLastError();
                 if (e != cudaSuccess) { rc = fail(CKV_ECUDA, "flush read sweep failed: %s", cudaGetErrorString(e)); break; }
             }
-            if (timed) cudaEventRecord(ev[2 * (size_t)(k - warmup)], s);
+            if (timed) record(ev[2 * (size_t)(k - warmup)]);
             for (int layer = 0; layer < c.num_layers && rc == CKV_OK; ++layer) {
                 const uint8_t *q = static_cast<const uint8_t *>(d_q) + q_layer * layer;
                 const uint8_t *kn = static_cast<const uint8_t *>(d_k_new) + kv_layer * layer;
@@ -686,19 +758,24 @@ int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch
                 uint8_t *o = static_cast<uint8_t *>(d_out) + q_layer * layer;
                 rc = decode_step(pool, layer, b, d_block_tables, d_seq_lens, q, kn, vn, o, stream);
             }
-            if (timed) cudaEventRecord(ev[2 * (size_t)(k - warmup) + 1], s);
+            if (timed) record(ev[2 * (size_t)(k - warmup) + 1]);
         }
         if (rc != CKV_OK) break;
         cudaError_t e = cudaStreamSynchronize(s);
         if (e != cudaSuccess) { rc = fail(CKV_ECUDA, "step_latency_sweep: synchronise failed: %s", cudaGetErrorString(e)); break; }
-        for (int k = 0; k < iters; ++k) cudaEventElapsedTime(&ms[k], ev[2 * (size_t)k], ev[2 * (size_t)k + 1]);
+        for (int k = 0; k < iters && rc == CKV_OK; ++k) {
+            const cudaError_t ce = cudaEventElapsedTime(&ms[k], ev[2 * (size_t)k], ev[2 * (size_t)k + 1]);
+            if (ce != cudaSuccess) rc = fail(CKV_ECUDA, "step_latency_sweep: cudaEventElapsedTime failed: %s", cudaGetErrorString(ce));
+        }
+        if (rc != CKV_OK) break;
         std::vector<float> sorted(ms);
         std::sort(sorted.begin(), sorted.end());
         const double med = (iters & 1) ? sorted[iters / 2] : 0.5 * (sorted[iters / 2 - 1] + sorted[iters / 2]);
         out_median_us[i] = med * 1000.0;
         out_min_us[i] = sorted[0] * 1000.0;
     }
-    for (auto &e : ev) cudaEventDestroy(e);
+    for (auto &e : ev)
+        if (e) cudaEventDestroy(e);
     if (rc != CKV_OK) return rc;
     return kv_check_status(pool, stream, nullptr);
 }
@@ -756,9 +833,15 @@ int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int3
     int device = -1;
     CKV_CUDA(cudaGetDevice(&device));
     if (device < 0 || device >= kMaxDevices) return fail(CKV_EINVAL, "decode_attention_noalloc: device ordinal %d not supported", device);
-    int cc_major = 0, sms = 0;
-    CKV_CUDA(cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, device));
-    CKV_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    static int cached_cc[kMaxDevices] = {}, cached_sms[kMaxDevices] = {};      // looked up on a device's first call
+    if (cached_sms[device] == 0) {
+        int cc = 0, n = 0;
+        CKV_CUDA(cudaDeviceGetAttribute(&cc, cudaDevAttrComputeCapabilityMajor, device));
+        CKV_CUDA(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device));
+        cached_cc[device] = cc;
+        cached_sms[device] = n;
+    }
+    const int cc_major = cached_cc[device], sms = cached_sms[device];
     if (cc_major != 10) return fail(CKV_ECUDA, "decode_attention_noalloc: device %d is sm_%dx; this library is built for sm_100a only", device, cc_major);
 
     const int warps = cfg->head_dim == 128 ? kWarps128 : kWarps64;
@@ -779,22 +862,8 @@ int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int3
     unsigned char *scratch = g_noalloc_ptr[device];
 
     // Tensor map over the caller's pool, built on the stack (a host-side encode, no allocation).
-    void *fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    cudaError_t ee = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-    if (ee != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
-        return fail(CKV_ECUDA, "decode_attention_noalloc: cuTensorMapEncodeTiled not available (%s)", cudaGetErrorString(ee));
     CUtensorMap tmap;
-    const cuuint64_t rows = (cuuint64_t)cfg->num_layers * cfg->num_pages * cfg->num_kv_heads * 32;
-    const cuuint64_t dims[2] = {(cuuint64_t)cfg->head_dim, rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)cfg->head_dim * 2};
-    const cuuint32_t box[2] = {64, 32};
-    const cuuint32_t estr[2] = {1, 1};
-    CUresult cr = reinterpret_cast<EncodeTiledFn>(fn)(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(d_pool),
-                                                      dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (cr != CUDA_SUCCESS) return fail(CKV_ECUDA, "decode_attention_noalloc: cuTensorMapEncodeTiled returned %d", (int)cr);
+    if (int32_t rc = encode_pool_map(cfg, d_pool, &tmap, "decode_attention_noalloc")) return rc;
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // The scratch keeps whatever the previous call left: the status word and the arrival counters

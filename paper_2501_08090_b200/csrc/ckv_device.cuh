@@ -162,6 +162,9 @@ struct GatherParams {
 
 __global__ void host_gather_kernel(const GatherParams p)
 {
+    // the attention kernel that follows may become resident right away; it waits for this grid
+    // before it reads anything
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const size_t tid = blockIdx.x * (size_t)blockDim.x + threadIdx.x, nthr = (size_t)gridDim.x * blockDim.x;
 #pragma unroll
     for (int a = 0; a < 5; ++a) {
@@ -348,13 +351,14 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 
 // Wait for a phase of an mbarrier, giving up after kWaitLimitNs.  Returns false when it gave up;
 // the status word is flagged and the caller stops working.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t *status)
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t *status,
+                                                  unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer_ns();
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (global_timer_ns() - t0 > kWaitLimitNs) {
+        if (global_timer_ns() - t0 > limit_ns) {
             atomicOr(status, kStatusWaitLimit);
             return false;
         }
@@ -522,7 +526,8 @@ struct AttnParams {
     int32_t layer_page_base;        // layer * num_pages
     int32_t num_spans;
     int32_t q_len;                  // new tokens per request in this step (1 for plain decode)
-    int32_t early_loads;            // the first tile loads may be issued before the dependency wait (fused step only)
+    int32_t early_loads;            // > 0: the first tile loads may be issued before the dependency wait (fused step only);
+                                    // < 0: even seq_lens and the tables come from the preceding kernel: wait before the plan
     int32_t q_base, q_pass;         // this launch computes new tokens q_base .. q_base + q_pass - 1; q_pass*group <= 8
     float scale_log2;               // log2(e) / sqrt(d)
 };
@@ -811,6 +816,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         fence_proxy_async();
     }
     __syncwarp();
+    if (p.early_loads < 0) grid_dependency_wait();
 
     // ---- plan: where does this warp's span start?
     // Nothing read up to the dependency wait below is written by the preceding kernel of a decode
@@ -954,7 +960,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     // hold a position >= L-2 therefore stay behind the dependency wait.  The dependents of this
     // kernel are released only after the wait, so a kernel's early loads overlap its immediate
     // predecessor and nothing older.
-    const bool early = p.k_new != nullptr && p.early_loads != 0;
+    const bool early = p.k_new != nullptr && p.early_loads > 0;
     if (early) {
         inputs_ready = false;
         while (issued < NS && more_to_issue && ic.tile < (ic.L - 2) / kTileTokens) issue_next();
@@ -1440,6 +1446,28 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         p.trace[span * 8 + 7] = n_pieces;
 #endif
     }
+}
+
+// ------------------------------------------------------------------------------------------
+// Self-test of the give-up path of the bounded waits.  One warp waits, with the same routine the
+// attention kernel uses but a caller-given limit, for a phase of an mbarrier that nothing will ever
+// complete: no copy is issued and nobody arrives.  When the limit runs out the routine flags the
+// status word and returns, and the warp leaves an arrival counter half-way, as an attention warp
+// that gave up in the middle of a merge would.  Nothing here can fault or hang: the only loop is
+// the bounded one.
+// ------------------------------------------------------------------------------------------
+__global__ void wait_limit_selftest_kernel(uint32_t *status, int32_t *arrivals, unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long bar_storage;
+    const uint32_t bar = smem_u32(&bar_storage);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    bool ok = mbar_wait_bounded(bar, 0, status, limit_ns);      // phase 0 never completes
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok && threadIdx.x == 0) atomicAdd(arrivals, 1);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -83,6 +83,30 @@ def test_mixed_sweep_full_batch_and_nested_prefixes():
     kp.close()
 
 
+def test_mixed_sweep_through_decode_step_the_call_the_sweep_times():
+    """step_latency_sweep and bench.py time decode_step (append + attention in one kernel): the full
+    batch of 512 and the nested prefixes through that call, sampled rows against the oracle, sampled
+    pages bit-exact."""
+    w, lens, npg, bt, kp, pool, q, k, v, out = _device_workload("mixed_sweep")
+    rows = _pick(lens, 14, seed=4, always=(0, 1, 2, 3, 7, 15, 31))
+    sub_pool_ref, ref = _oracle_on_sample(w, pool, bt, lens, rows, 0, q, k, v)
+    btd, sld = torch.from_numpy(bt).cuda(), torch.from_numpy(lens).cuda()
+    for B in (512, 1, 2, 4, 8, 16, 32, 64, 128, 256):
+        out.fill_(float("nan"))
+        kp.decode_step(0, btd[:B], sld[:B], q[0][:B], k[0][:B], v[0][:B], out[0][:B])
+        assert kp.check_status() == 0
+        got = dev_to_bits(out[0])
+        inside = [i for i, r in enumerate(rows) if r < B]
+        assert inside
+        assert_close(got[[rows[i] for i in inside]], ref[inside], "mixed_sweep decode_step B=%d" % B)
+        assert torch.isfinite(out[0][:B].float()).all()
+        assert np.isnan(widen(got[B:])).all()
+        if B == 512:
+            sub_after, _, _, _ = compact_requests(pool, bt, lens, rows, 0)
+            assert np.array_equal(sub_after, sub_pool_ref)
+    kp.close()
+
+
 def test_llama70b_two_layers_append_touches_exactly_the_target_rows():
     """Reduced-layer variant where a second copy of the pool fits: global untouched-bytes check."""
     w, lens, npg, bt, kp, pool, q, k, v, out = _device_workload("llama70b_full", num_layers=2)
@@ -109,14 +133,14 @@ def test_llama70b_two_layers_append_touches_exactly_the_target_rows():
 def test_llama70b_all_80_layers_sampled_parity():
     w, lens, npg, bt, kp, pool, q, k, v, out = _device_workload("llama70b_full")
     assert w.num_layers == 80 and pool.numel() * 2 > 79e9
-    layers = (0, 1, 39, 79)
-    rows = _pick(lens, 4, seed=5)
+    layers = (0, 1, 13, 27, 39, 52, 66, 79)                                # every request of the batch on these ...
+    rows = list(range(lens.size))
     refs = {layer: _oracle_on_sample(w, pool, bt, lens, rows, layer, q, k, v) for layer in layers}
     btd, sld = torch.from_numpy(bt).cuda(), torch.from_numpy(lens).cuda()
     for layer in range(w.num_layers):                                      # one whole decode iteration
         kp.decode_step(layer, btd, sld, q[layer], k[layer], v[layer], out[layer])
     assert kp.check_status() == 0
-    assert torch.isfinite(out.float()).all()
+    assert torch.isfinite(out.float()).all()                               # ... and nothing non-finite on the other 72
     for layer in layers:
         sub_ref, ref = refs[layer]
         sub_after, _, _, _ = compact_requests(pool, bt, lens, rows, layer)

@@ -446,13 +446,18 @@ def test_skewed_long_context_full_parity():
 
 # --------------------------------------------------------------------------- host-buffer entry and sweep
 
-@pytest.mark.parametrize("pinned", [True, False])
-def test_decode_step_host_matches_oracle(pinned):
-    """Pinned buffers take the zero-copy route (gather kernel in, output rows written straight to
-    the host buffer), pageable ones the copy route; both must give the oracle's step."""
-    h = wl.host_inputs(wl.workload("tiny"))
+@pytest.mark.parametrize("pinned,route,launches", [(True, "auto", 2), (True, "staged", 2), (True, "direct", 1),
+                                                   (True, "copy", 1), (False, "auto", 1), (False, "direct", 1)])
+def test_decode_step_host_matches_oracle(pinned, route, launches):
+    """Pinned buffers take a zero-copy route (staged through a gather kernel, or read directly by
+    the attention kernel; output rows written straight to the host buffer), pageable ones the copy
+    route whatever was asked for; every route must give the oracle's step."""
+    from paper_2501_08090_b200 import binding as b
+    h = custom_inputs([700, 90, 2000, 64, 1500, 333, 800, 16, 4000], 8, 2, 128, seed=67)
     ref_pool, ref_out = oracle_step(h)
     ds = make_device_step(h)
+    ds.pool.set_host_route({"auto": b.HOST_ROUTE_AUTO, "staged": b.HOST_ROUTE_STAGED, "direct": b.HOST_ROUTE_DIRECT,
+                            "copy": b.HOST_ROUTE_COPY}[route])
     host = lambda a: torch.from_numpy(np.ascontiguousarray(a).copy())
     pin = (lambda a: host(a).pin_memory()) if pinned else host
     q = pin(h.q[0].view(np.int16)).view(torch.bfloat16)
@@ -460,12 +465,19 @@ def test_decode_step_host_matches_oracle(pinned):
     v = pin(h.v_new[0].view(np.int16)).view(torch.bfloat16)
     out = torch.zeros_like(q)
     out = out.pin_memory() if pinned else out
+    bt, sl = pin(h.block_tables), pin(h.seq_lens)
     n0 = ds.pool.launch_count()
-    ds.pool.decode_step_host(0, pin(h.block_tables), pin(h.seq_lens), q, k, v, out)
-    assert ds.pool.launch_count() - n0 == (2 if pinned else 1)
+    ds.pool.decode_step_host(0, bt, sl, q, k, v, out)
+    assert ds.pool.launch_count() - n0 == launches
     assert ds.pool.check_status() == 0
     assert np.array_equal(dev_to_bits(ds.pool.pool), ref_pool)
-    assert_close(dev_to_bits(out), ref_out, "decode_step_host pinned=%s" % pinned)
+    assert_close(dev_to_bits(out), ref_out, "decode_step_host pinned=%s route=%s" % (pinned, route))
+    # the pre-marshalled form issues the same step (same lengths: the append rewrites the same rows)
+    out.zero_()
+    ds.pool.host_step_call(0, bt, sl, q, k, v, out)()
+    assert ds.pool.check_status() == 0
+    assert_close(dev_to_bits(out), ref_out, "host_step_call pinned=%s route=%s" % (pinned, route))
+    ds.pool.close()
 
 
 def test_step_latency_sweep_runs_nested_prefixes_and_counts_launches():

@@ -4,8 +4,9 @@ Some users of this library have nowhere to put split-KV partials: an engine that
 device memory to the KV pool at start-up, a plugin under a framework that owns the allocator, a
 latency-critical loop that cannot take cudaMalloc's device-wide synchronisation.  For them the
 partials live in a fixed array inside the library.  This test drives that entry point through the
-C ABI and checks it against decode_attention (which uses a caller-provided workspace) on two
-calls in a row -- the second call finds the array as the first one left it.
+C ABI and checks it against the fp64 oracle and against decode_attention (which uses a
+caller-provided workspace) on two calls in a row -- the second call finds the array as the first
+one left it.
 
 Collected last on purpose (file name), so a run that stops at the first failure has already run
 every other test.
@@ -16,9 +17,11 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import oracle
+from oracle.oracle import PoolShape
 from paper_2501_08090_b200 import workloads as wl
 
-from helpers import ATOL, RTOL, bits_to_dev, dev_to_bits, widen
+from helpers import ATOL, RTOL, assert_close, bits_to_dev, dev_to_bits, widen
 
 pytestmark = pytest.mark.gpu
 
@@ -33,7 +36,12 @@ def _inputs(lens, seed, Hq=32, Hkv=8, d=128):
                 q=wl.normal_bf16((B, Hq, d), seed, 2))
 
 
-def _run_both(b, inp, num_spans=0):
+def _oracle(inp):
+    sh = PoolShape(1, inp["npg"], inp["Hq"], inp["Hkv"], 16, inp["d"])
+    return oracle.decode_attention(inp["pool"].reshape(-1), sh, 0, inp["bt"], inp["lens"], inp["q"])
+
+
+def _run_both(b, inp, num_spans=0, sync=True):
     """(output of decode_attention, output of decode_attention_noalloc) as float64 arrays."""
     B = inp["lens"].size
     cfg = b.make_config(1, inp["Hq"], inp["Hkv"], inp["d"], inp["npg"], inp["bt"].shape[1], B)
@@ -51,8 +59,11 @@ def _run_both(b, inp, num_spans=0):
     assert kp.check_status() == 0
     kp.close()
 
-    bits = b.decode_attention_noalloc(cfg, pool, 0, bt, sl, q, got, num_spans=num_spans)
+    bits = b.decode_attention_noalloc(cfg, pool, 0, bt, sl, q, got, num_spans=num_spans, sync=sync)
     assert bits == 0
+    if not sync:
+        torch.cuda.synchronize()                   # the call only enqueued work
+    assert_close(dev_to_bits(got), _oracle(inp), "decode_attention_noalloc against the oracle")
     return widen(dev_to_bits(ref)), widen(dev_to_bits(got))
 
 
@@ -70,6 +81,9 @@ def test_noalloc_matches_decode_attention_on_two_calls_in_a_row():
     # and once more with a narrow partition and the small head size
     third = _inputs([300, 77, 1000], seed=903, Hq=4, Hkv=1, d=64)
     ref, got = _run_both(b, third, num_spans=7)
+    assert np.all(np.abs(got - ref) <= ATOL + RTOL * np.abs(ref))
+    # enqueue-only form (no status pointer): the caller synchronises
+    ref, got = _run_both(b, second, sync=False)
     assert np.all(np.abs(got - ref) <= ATOL + RTOL * np.abs(ref))
 
 

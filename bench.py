@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on the headline
 # workload, from the ncu capture summarised in profiles/paged_decode_attn_llama8b_b64.md.  Set to
 # None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES = None       # dram read + write per launch of the attention kernel (ncu); None: not captured for this kernel
+NCU_TRAFFIC_BYTES = 573.3e6    # dram read + write per launch of the attention kernel, mean of 2 captured launches (profiles/paged_decode_attn_llama8b_b64.md)
 
 
 # ------------------------------------------------------------------------------- clocks
@@ -349,7 +349,7 @@ def run_ours(args) -> None:
     rank, world, local = dist_setup(args.gpus)
     dev = torch.device("cuda", local if world > 1 else 0)
     name = args.workload or HEADLINE
-    dw = DeviceWorkload(name, dev, seed_offset=rank, num_layers=args.layers)
+    dw = DeviceWorkload(name, dev, seed_offset=rank, batch=args.batch, num_layers=args.layers)
     w = dw.w
     K, W = args.steps, max(args.warmup, 3)
 
@@ -418,12 +418,16 @@ def run_ours(args) -> None:
         for _ in range(n):
             for call in host_calls:
                 call()
-    e2e_steps(3)
+    e2e_steps(50)
     barrier(world)
-    t0 = time.perf_counter()
-    e2e_steps(E)
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
+    chunks = []
+    for _ in range(5):                                  # E steps in five chunks; the median chunk is reported
+        t0 = time.perf_counter()
+        e2e_steps(E // 5)
+        torch.cuda.synchronize()
+        chunks.append(time.perf_counter() - t0)
+    E = 5 * (E // 5)
+    e2e_s = statistics.median(chunks) * 5
     e2e_ms_max, e2e_bytes = reduce_max_sum(e2e_s * 1e3, float(dw.bytes["total"]) * E, world)
     e2e = {"value": e2e_bytes / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d * w.num_layers,
            "d2h_bytes_per_step": d2h * w.num_layers, "steps": E, "us_per_step": e2e_ms_max / E * 1e3,
@@ -714,6 +718,7 @@ def main() -> None:
     ap.add_argument("--no-sweep", action="store_true", help="skip the batch-size latency sweep")
     ap.add_argument("--workload", default=None, help="time another workload than the headline one (profiling runs)")
     ap.add_argument("--layers", type=int, default=None, help="number of layers of that workload to make resident")
+    ap.add_argument("--batch", type=int, default=None, help="take only the first BATCH requests of that workload (profiling runs)")
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip timing the CPU oracle (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -418,7 +418,7 @@ def run_ours(args) -> None:
         for _ in range(n):
             for call in host_calls:
                 call()
-    e2e_steps(50)
+    e2e_steps(E)                                        # warm-up: the host side takes a few hundred calls to settle
     barrier(world)
     chunks = []
     for _ in range(5):                                  # E steps in five chunks; the median chunk is reported

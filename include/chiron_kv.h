@@ -161,7 +161,7 @@ int32_t decode_attention_multi(ckv_pool *pool, int32_t layer, int32_t batch, int
  * inspection (runs a small kernel and synchronises `stream`; decode_attention itself derives the
  * same partition inside its attention kernel and launches no plan kernel).  A "tile" is 32
  * consecutive tokens of one (request, KV head).  Work is laid out on an axis of units,
- * request-major then KV head: each (request, KV head) contributes CKV_PIECE_COST_TILES (2)
+ * request-major then KV head: each (request, KV head) contributes CKV_PIECE_COST_TILES (3)
  * overhead units followed by one unit per tile.  Span s -- the work of one warp -- owns the tiles
  * whose units fall in [s*units_per_span, min((s+1)*units_per_span, total_units)).
  *   h_header[4]   : total_units, units_per_span, num_spans, number of spans with a non-empty range

@@ -19,7 +19,7 @@ LIBRARY = os.path.join(_HERE, "libchiron_kv.so")
 CKV_OK, CKV_EINVAL, CKV_ENOMEM, CKV_ECUDA, CKV_EBOUNDS, CKV_ETIMEOUT = 0, -1, -2, -3, -4, -5
 STATUS_BAD_LENGTH, STATUS_BAD_PAGE, STATUS_WAIT_LIMIT = 1, 2, 4
 HOST_ROUTE_AUTO, HOST_ROUTE_STAGED, HOST_ROUTE_DIRECT, HOST_ROUTE_COPY = 0, 1, 2, 3
-TILE_TOKENS, PIECE_COST_TILES = 32, 2      # the plan's tile size and per-piece overhead units
+TILE_TOKENS, PIECE_COST_TILES = 32, 3      # the plan's tile size and per-piece overhead units
 
 EXPORTS = (
     "kv_pool_bytes", "kv_workspace_bytes", "kv_pool_create", "kv_pool_destroy", "kv_append",

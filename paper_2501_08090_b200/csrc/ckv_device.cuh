@@ -30,11 +30,11 @@ constexpr unsigned long long kWaitLimitNs = 1000000000ull;   // bound of every d
 
 // The split-KV partition.  Work is laid out on one axis of "units", request-major, then kv head:
 // every (request, kv head) contributes kPieceCostTiles overhead units (the fixed cost of starting,
-// finishing and merging a piece, measured at about two tiles' worth of time) followed by one unit
+// finishing and merging a piece: three tiles' worth of time balanced best across the workloads) followed by one unit
 // per tile.  Span s owns the tiles whose units fall in [s*q, min((s+1)*q, total)), q =
 // ceil(total/spans), so spans that hold many short (request, kv head) pieces get fewer tiles.
 #ifndef CKV_PIECE_COST_TILES
-#define CKV_PIECE_COST_TILES 2
+#define CKV_PIECE_COST_TILES 3
 #endif
 constexpr int kPieceCostTiles = CKV_PIECE_COST_TILES;
 

@@ -110,7 +110,7 @@ def compact_requests(pool_dev: torch.Tensor, bt: np.ndarray, lens: np.ndarray, r
 
 # ----------------------------------------------------------------------------- the plan's spec
 
-def expected_plan(lens_np, Hkv, C, cost=2):
+def expected_plan(lens_np, Hkv, C, cost=3):
     """The partition spec restated: `cost` overhead units then one unit per 32-token tile for every
     (request, kv head); span s owns the tiles whose units lie in [s*q, (s+1)*q)."""
     tiles = (lens_np.astype(np.int64) + 31) // 32
@@ -133,7 +133,7 @@ def expected_plan(lens_np, Hkv, C, cost=2):
     return total, q, starts.astype(np.int32)
 
 
-def covered_tiles(lens_np, Hkv, C, cost=2, counts=None):
+def covered_tiles(lens_np, Hkv, C, cost=3, counts=None):
     """All (request, kv head, tile) triples the spans of the spec visit, in order.
     If `counts` is a list, the number of tiles of every span is appended to it."""
     tiles = (lens_np.astype(np.int64) + 31) // 32

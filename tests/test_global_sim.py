@@ -266,3 +266,27 @@ def test_bad_inputs_are_rejected(b):
         b.global_simulate(b.SimConfig(**base_config()), ok[0], [0, 2], *ok[2:])   # unknown kind
     with pytest.raises(b.CkvError):
         b.global_simulate(b.SimConfig(**base_config(policy=7)), *ok)
+
+
+def test_random_configurations_event_for_event(b):
+    """Thirty random instance models, bands, start-up delays, group counts and traces (including pools
+    that start empty, zero floors and tiny slot counts): the library and the oracle's event loop must
+    produce the same events, and both must terminate."""
+    rng = np.random.default_rng(77)
+    for trial in range(30):
+        n = int(rng.integers(20, 220))
+        kw = base_config(
+            slots_interactive=int(rng.integers(1, 6)), slots_batch=int(rng.integers(1, 12)),
+            rate_interactive=float(rng.uniform(5, 40)), rate_batch=float(rng.uniform(2, 20)),
+            startup_s=float(rng.choice([0.0, 3.0, 20.0])), tick_s=float(rng.choice([1.0, 5.0, 13.0])),
+            theta=float(rng.choice([0.25, 1.0 / 3.0, 0.5, 0.8])), delta=float(rng.choice([0.0, 0.05, 0.15])),
+            floor_instances=int(rng.integers(0, 3)), initial_instances=int(rng.integers(0, 5)),
+            max_batch_instances=int(rng.integers(0, 6)), groups_k=int(rng.integers(1, 5)),
+            z=float(rng.choice([0.0, 1.0, 2.33])), policy=int(rng.integers(0, 2)),
+            horizon_s=float(rng.choice([0.0, 0.0, 150.0])))
+        arrival, kind, tokens, slo = wl.request_trace(n, float(rng.uniform(0.5, 6.0)), float(rng.choice([1.0, 3.0])),
+                                                      float(rng.uniform(0.0, 1.0)), 1000 + trial,
+                                                      batch_ttft_s=float(rng.choice([30.0, 200.0])))
+        slo = np.where((kind == 1) & (np.arange(n) % 4 == 0), slo / 3.0, slo)
+        got, want = run_both(b, kw, (arrival, kind, tokens, slo))
+        assert_same_run(got, want)

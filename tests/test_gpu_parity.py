@@ -329,9 +329,10 @@ def test_read_probe_streams_the_batch_and_reports_bad_pages():
 @pytest.mark.parametrize("Hq,Hkv", [(4, 1), (8, 1), (8, 2)])
 def test_every_merge_stage_matches_oracle(Hq, Hkv):
     """One long context cut into C spans exercises each way partials are merged: inside one CTA
-    through shared memory (C <= 4 spans), two CTAs with the later one merging from its registers
-    (5..8), a flat merge of up to 24 CTA partials, and the two-level merge beyond that -- with a
-    short request behind it so that the last span also holds a whole (request, kv head)."""
+    through shared memory (C <= 4 spans), two CTAs with the later one fetching the other's partial
+    (5..8), a flat merge of up to 24 CTA partials (in several rounds where they do not fit the ring
+    at once: 8 columns, C = 96), and the two-level merge beyond that -- with a short request
+    behind it so that the last span also holds a whole (request, kv head)."""
     h = custom_inputs([9000, 70], Hq, Hkv, 128, seed=500 + Hq + Hkv)
     ref_pool, ref_out = oracle_step(h)
     for fused in (False, True):
@@ -344,7 +345,7 @@ def test_every_merge_stage_matches_oracle(Hq, Hkv):
 
 def test_results_are_bit_identical_from_run_to_run():
     """Which warp or CTA arrives last at a merge differs from launch to launch; the bits of the
-    output must not (partials are folded in a fixed order, and the two-CTA merge is symmetric)."""
+    output must not (partials are folded in the order of their index, whoever does the folding)."""
     rng = np.random.default_rng(5)
     lens = rng.integers(300, 3000, size=48).tolist() + [20000]
     h = custom_inputs(lens, 8, 2, 128, seed=77)

@@ -849,7 +849,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     SpanCursor ic;
     ic.r = st.r; ic.h = st.h; ic.tile = st.tile; ic.L = st.L; ic.tiles = st.tiles_r; ic.v = st.v;
     bool more_to_issue = true;                   // the issue cursor still points at a tile of this span
-    int issued = 0;
+    int issued = 0, i_slot = 0;                  // i_slot = issued % NS
     bool alive = true;
     auto table_row = [&](int r) { return p.block_tables + (size_t)r * p.max_pages_per_req; };
     auto load_chunk = [&](int r, int chunk) -> int {
@@ -908,7 +908,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         const int np = min(kPagesPerTile, n_pages - ic.tile * kPagesPerTile);
         const int pg = lane / Lay::kHalves, hf = lane % Lay::kHalves;
         int page = __shfl_sync(0xffffffffu, cur_val, ((ic.tile % kTilesPerChunk) * kPagesPerTile + pg) & 31);
-        const int slot = issued % NS;
+        const int slot = i_slot;
+        if (++i_slot == NS) i_slot = 0;
         // The stage's previous contents were read by this warp's ldmatrix instructions, whose results
         // have all been consumed by MMAs earlier in program order, so the reads are complete.
         if (lane == 0) mbar_arrive_expect_tx(bars + slot * 8, np * Lay::kPageBytes);
@@ -994,6 +995,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     }
 
     int done = 0;                                // tiles computed (or skipped after a wait gave up)
+    int c_slot = 0;                              // done % NS and the parity of done / NS, kept without divisions
+    uint32_t c_phase = 0;
     int landed = 0;                              // tiles whose copies were seen to complete
     bool more_to_compute = true;
     unsigned long long t_wait = 0, t_between = 0, t_piece_end = 0;
@@ -1022,12 +1025,14 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         for (int dt = 0; dt < Lay::kDTiles; ++dt) o[dt][0] = o[dt][1] = o[dt][2] = o[dt][3] = 0.f;
 
         for (int ti = piece_tile0; ti < piece_tile0 + n; ++ti, ++done) {
-            const int slot = done % NS;
+            const int slot = c_slot;
+            const uint32_t phase = c_phase;
+            if (++c_slot == NS) { c_slot = 0; c_phase ^= 1u; }
             if (alive) {
 #ifdef CKV_TRACE_WAITS
                 const unsigned long long w0 = global_timer_ns();
 #endif
-                alive = mbar_wait_bounded(bars + slot * 8, (done / NS) & 1, p.status);
+                alive = mbar_wait_bounded(bars + slot * 8, phase, p.status);
                 alive = __all_sync(0xffffffffu, alive);
 #ifdef CKV_TRACE_WAITS
                 t_wait += global_timer_ns() - w0;
@@ -1110,18 +1115,26 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
                 }
             }
 
-            // ---- online softmax in the log2 domain
+            // ---- online softmax in the log2 domain.  Scores stay unscaled: the scale rides in the
+            // FMA that forms the exponent, and a maximum is scaled once (the scale is positive).
+            if (!full_tile) {
+#pragma unroll
+                for (int mt = 0; mt < kPagesPerTile; ++mt) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int tok = mt * kPageSize + (lane >> 2) + (i >= 2 ? 8 : 0);
+                        if (!(tok < ((i & 1) ? lim1 : lim0))) s[mt][i] = -INFINITY;      // selected, never multiplied
+                    }
+                }
+            }
             float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
             for (int mt = 0; mt < kPagesPerTile; ++mt) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int tok = mt * kPageSize + (lane >> 2) + (i >= 2 ? 8 : 0);
-                    const float t = (full_tile || tok < ((i & 1) ? lim1 : lim0)) ? s[mt][i] * p.scale_log2 : -INFINITY;
-                    s[mt][i] = t;
-                    if (i & 1) mx1 = fmaxf(mx1, t); else mx0 = fmaxf(mx0, t);
-                }
+                mx0 = fmaxf(mx0, fmaxf(s[mt][0], s[mt][2]));
+                mx1 = fmaxf(mx1, fmaxf(s[mt][1], s[mt][3]));
             }
+            mx0 *= p.scale_log2;
+            mx1 *= p.scale_log2;
             // The reference a column's exponentials are taken against only has to be near its maximum:
             // it moves (with the reduction across lanes and the rescale that this costs) only when
             // some score of the tile exceeds it by more than 2^8.
@@ -1153,8 +1166,8 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             uint32_t pb[kPagesPerTile][2];
 #pragma unroll
             for (int mt = 0; mt < kPagesPerTile; ++mt) {
-                const float p0 = fast_exp2(s[mt][0] - mn0), p1 = fast_exp2(s[mt][1] - mn1);
-                const float p2 = fast_exp2(s[mt][2] - mn0), p3 = fast_exp2(s[mt][3] - mn1);
+                const float p0 = fast_exp2(fmaf(s[mt][0], p.scale_log2, -mn0)), p1 = fast_exp2(fmaf(s[mt][1], p.scale_log2, -mn1));
+                const float p2 = fast_exp2(fmaf(s[mt][2], p.scale_log2, -mn0)), p3 = fast_exp2(fmaf(s[mt][3], p.scale_log2, -mn1));
                 l0 += p0 + p2;
                 l1 += p1 + p3;
                 pb[mt][0] = movmatrix_trans(pack_bf16x2(p0, p1));       // tokens 0..7 of the page

@@ -1422,21 +1422,29 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
         }
     }
 
-    // ---- run the grid-stage jobs: both fetches first, so that their round trips overlap
+    // ---- run the grid-stage jobs.  The rounds of a fold (and with them its rounding) must not depend
+    // on which warp happened to come last, so a job's round size is a function of its own size only:
+    // two jobs that each fit half the ring in one round share it, their fetches in flight together;
+    // otherwise a job has the whole ring and the second one starts after the first.
     if (alive && n_jobs > 0) {
-        const int region = NS * Lay::kStageBytes / n_jobs;
-        fence_proxy_async();                      // partials written through the generic proxy, read by bulk copies
+        const int whole = NS * Lay::kStageBytes;
+        const bool share = n_jobs == 2 && max(jobs[0].n, jobs[1].n) <= (whole / 2) / part_bytes;
 #pragma unroll 1
-        for (int i = 0; i < n_jobs; ++i) {
-            jobs[i].base = ring + i * region;
-            jobs[i].cap = min(32, region / part_bytes);
-            jobs[i].bar = bars + i * 8;
-            jobs[i].uses = bar_uses[i];
-            fold_fetch<D>(jobs[i], fc, 0);
+        for (int s = 0; s < 2 * n_jobs && alive; ++s) {
+            const int i = share ? (s & 1) : (s >> 1);
+            const bool fetch = share ? s < 2 : !(s & 1);
+            if (fetch) {
+                jobs[i].base = ring + (share ? i * (whole / 2) : 0);
+                jobs[i].cap = min(32, (share ? whole / 2 : whole) / part_bytes);
+                jobs[i].bar = bars + i * 8;
+                jobs[i].uses = bar_uses[i];
+                fence_proxy_async();              // generic-proxy accesses (the partials' stores, an earlier job's reads) before the copies
+                __syncwarp();
+                fold_fetch<D>(jobs[i], fc, 0);
+            } else if (fold_finish<D>(jobs[i], fc) < 0) {
+                alive = false;
+            }
         }
-#pragma unroll 1
-        for (int i = 0; i < n_jobs && alive; ++i)
-            if (fold_finish<D>(jobs[i], fc) < 0) alive = false;
     }
 
     // Do not leave while copies into this warp's ring may still be in flight (only after a wait gave up).

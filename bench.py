@@ -451,6 +451,7 @@ def run_ours(args) -> None:
     e2e_ms_max, e2e_bytes = reduce_max_sum(e2e_s * 1e3, float(dw.bytes["total"]) * E, world)
     e2e = {"value": e2e_bytes / (e2e_ms_max * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d * w.num_layers,
            "d2h_bytes_per_step": d2h * w.num_layers, "steps": E, "us_per_step": e2e_ms_max / E * 1e3,
+           "chunk_us_per_step": [round(c / (E // 5) * 1e6, 1) for c in chunks],
            "route": "decode_step_host, pinned host buffers: gather kernel in, output rows written to host memory by the "
                     "attention kernel, one synchronise per step"}
 

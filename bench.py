@@ -406,6 +406,18 @@ def run_ours(args) -> None:
                 "isolated": {"us_per_launch": attn_ms / attn_n * 1e3, "achieved": isolated, "frac": isolated / peak,
                              "timing": "events around every launch, no overlap between launches"}}
 
+    # ---- the same K steps in plain stream order (no programmatic dependent launch): every launch starts
+    # after the one before has ended, with nothing but the stream's own gap between them
+    dw.kp.set_overlap(False)
+    dw.run_steps(W)
+    ser_ms, _ = timed_region(lambda: dw.run_steps(K), world, dev.index or 0)
+    dw.kp.set_overlap(True)
+    dw.kp.check_status()
+    ser_us = ser_ms * 1e3 / (K * w.num_layers)
+    roofline["serialized"] = {"us_per_launch": ser_us, "achieved": attn_bytes / (ser_us * 1e-6) / 1e9,
+                              "frac": attn_bytes / (ser_us * 1e-6) / 1e9 / peak,
+                              "timing": "K steps back to back in plain stream order, launches not overlapped"}
+
     # ---- the read probe: the same tiles through the same rings, no arithmetic: the practical ceiling
     def probe_steps(n):
         for _ in range(n):
@@ -470,6 +482,7 @@ def run_ours(args) -> None:
         "kv_gbs": kv_all / (ms_max * 1e-3) / 1e9, "frac_of_8TBs": value / NORMALISED_TO_TBS,
         # the same launch standing alone (events around every launch: what an engine that runs other
         # kernels between attention launches sees)
+        "serialized_us_per_launch": ser_us,
         "isolated_us_per_launch": attn_ms / attn_n * 1e3, "isolated_frac_of_8TBs": isolated / (NORMALISED_TO_TBS * 1e3),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches_all), "roofline": roofline,
     }

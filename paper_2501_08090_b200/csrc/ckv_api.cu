@@ -79,7 +79,7 @@ bool config_ok(const ckv_config *c, const char **why)
 }
 
 struct WorkspaceLayout {
-    size_t status, header, span_start, part_acc, part_ml, arrivals, trace;
+    size_t status, header, span_start, part, arrivals, trace;
     size_t st_tables, st_lens, st_q, st_k, st_v, st_out;
     size_t total;
 };
@@ -93,8 +93,7 @@ WorkspaceLayout carve(const ckv_config &c)
     w.status = take(256);
     w.header = take(sizeof(ckv::PlanHeader));
     w.span_start = take(sizeof(int4) * ckv::kMaxSpans);
-    w.part_acc = take(sizeof(float) * 2 * ckv::kMaxSpans * ckv::kMaxGroup * c.head_dim);
-    w.part_ml = take(sizeof(float) * 2 * ckv::kMaxSpans * 2 * ckv::kMaxGroup);
+    w.part = take(sizeof(float) * 2 * ckv::kMaxSpans * (2 * ckv::kMaxGroup + ckv::kMaxGroup * c.head_dim));
     w.arrivals = take(sizeof(int32_t) * ckv::kMaxSpans);
     w.trace = take(sizeof(unsigned long long) * 8 * ckv::kMaxSpans);
     w.st_tables = take(sizeof(int32_t) * (size_t)c.max_batch * c.max_pages_per_req);
@@ -238,10 +237,9 @@ constexpr size_t kNaStatus = 0;                                                 
 constexpr size_t kNaArrivals = 256;                                                   // int32 [640]
 constexpr size_t kNaSpanStart = kNaArrivals + sizeof(int32_t) * kNoAllocMaxSpans;     // int4 [640]
 constexpr size_t kNaTrace = kNaSpanStart + sizeof(int4) * kNoAllocMaxSpans;           // u64 [640][8]
-constexpr size_t kNaPartMl = kNaTrace + sizeof(unsigned long long) * 8 * kNoAllocMaxSpans;
-constexpr size_t kNaPartAcc = kNaPartMl + sizeof(float) * 2 * kNoAllocMaxSpans * 2 * ckv::kMaxGroup;
-constexpr size_t kNoAllocScratchBytes = kNaPartAcc + sizeof(float) * 2 * kNoAllocMaxSpans * ckv::kMaxGroup * 128;
-static_assert(kNaSpanStart % 16 == 0 && kNaTrace % 8 == 0 && kNaPartMl % 16 == 0 && kNaPartAcc % 256 == 0,
+constexpr size_t kNaPart = kNaTrace + sizeof(unsigned long long) * 8 * kNoAllocMaxSpans;   // partial slots
+constexpr size_t kNoAllocScratchBytes = kNaPart + sizeof(float) * 2 * kNoAllocMaxSpans * (2 * ckv::kMaxGroup + ckv::kMaxGroup * 128);
+static_assert(kNaSpanStart % 16 == 0 && kNaTrace % 8 == 0 && kNaPart % 256 == 0,
               "sub-buffers of the static scratch must keep their natural alignment");
 
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
@@ -466,8 +464,7 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
     ap.v_new = static_cast<const uint4 *>(d_v_new);
     ap.pool_layer = d_k_new ? reinterpret_cast<uint4 *>(pool->d_pool + (size_t)c.num_pages * c.num_kv_heads * 2 * c.page_size * c.head_dim * 2 * layer)
                             : nullptr;
-    ap.part_acc = pool->wsp<float>(pool->ws.part_acc);
-    ap.part_ml = pool->wsp<float>(pool->ws.part_ml);
+    ap.part = pool->wsp<float>(pool->ws.part);
     ap.arrivals = pool->wsp<int32_t>(pool->ws.arrivals);
     ap.span_start = pool->wsp<int4>(pool->ws.span_start);
     ap.trace = pool->wsp<unsigned long long>(pool->ws.trace);
@@ -875,8 +872,7 @@ int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int3
     ap.seq_lens = d_seq_lens;
     ap.q = static_cast<const uint16_t *>(d_q);
     ap.out = static_cast<uint16_t *>(d_out);
-    ap.part_acc = reinterpret_cast<float *>(scratch + kNaPartAcc);
-    ap.part_ml = reinterpret_cast<float *>(scratch + kNaPartMl);
+    ap.part = reinterpret_cast<float *>(scratch + kNaPart);
     ap.arrivals = reinterpret_cast<int32_t *>(scratch + kNaArrivals);
     ap.span_start = reinterpret_cast<int4 *>(scratch + kNaSpanStart);
     ap.trace = reinterpret_cast<unsigned long long *>(scratch + kNaTrace);

@@ -515,8 +515,8 @@ struct AttnParams {
     const uint4 *k_new;             // bf16 [batch][Hkv][d]
     const uint4 *v_new;
     uint4 *pool_layer;
-    float *part_acc;                // [2*kMaxSpans][8][D]   two slots per CTA are used: 2*cta, 2*cta + 1
-    float *part_ml;                 // [2*kMaxSpans][16]  (m[8], l[8])
+    float *part;                    // [2*kMaxSpans][16 + 8*D]: a partial is (m[8], l[8]), then its rows [8][D];
+                                    //   two slots per CTA are used: 2*cta, 2*cta + 1
     int32_t *arrivals;              // [kMaxSpans], all zero between launches
     int4 *span_start;               // [kMaxSpans] what each span started at (diagnostic)
     unsigned long long *trace;      // [kMaxSpans][8] ns: start, first tile landed, last tile done, span done,
@@ -581,7 +581,7 @@ struct FoldJob {
     int n;                          // partials to fold, in this order
     int cap;                        // partials per round (shared-memory sources: n)
     // partial t of a round that starts at t0 sits in shared memory at base + (t - t0) * stride:
-    // rows of `pitch` floats, (m, l) at byte offset ml_off ...
+    // rows of `pitch` floats, (m, l) at byte offset ml_off (negative for a fetched partial) ...
     uint32_t base;
     int stride, pitch, ml_off;
     // ... except partial alt_t (if >= 0), which sits at alt_base
@@ -609,8 +609,7 @@ struct FoldJob {
 };
 
 struct FoldCtx {
-    float *part_acc;                // [slots][8][D]
-    float *part_ml;                 // [slots][16]
+    float *part;                    // [slots][16 + 8*D]: (m[8], l[8]), then rows [8][D]
     uint32_t *status;
     int ncols, lane;
     int out_off;                    // elements from a pair's first output row to this lane's first float4 piece
@@ -635,9 +634,8 @@ __device__ __forceinline__ void fold_fetch(const FoldJob j, const FoldCtx c, int
     __syncwarp();
     if (c.lane < cnt && t0 + c.lane != j.alt_t) {
         const int slot = j.slot_of(t0 + c.lane);
-        const uint32_t dst = j.base + c.lane * j.stride;
-        bulk_load_1d(dst, c.part_acc + (size_t)slot * kMaxGroup * D, row_bytes, j.bar);
-        bulk_load_1d(dst + j.ml_off, c.part_ml + slot * 2 * kMaxGroup, 64, j.bar);
+        const uint32_t dst = j.base - 64 + c.lane * j.stride;    // j.base is where the rows go; (m, l) sit in front of them
+        bulk_load_1d(dst, c.part + (size_t)slot * (2 * kMaxGroup + kMaxGroup * D), 64 + row_bytes, j.bar);   // (m, l) and the live rows: one copy
     }
 }
 
@@ -717,13 +715,14 @@ __device__ __forceinline__ int fold_finish(const FoldJob j, const FoldCtx c)
             }
         }
     } else {
-        float *rows = c.part_acc + (size_t)j.dst_slot * kMaxGroup * D + g * D + d0;
+        float *slot = c.part + (size_t)j.dst_slot * (2 * kMaxGroup + kMaxGroup * D);
+        float *rows = slot + 2 * kMaxGroup + g * D + d0;
 #pragma unroll
         for (int q = 0; q < 8; ++q)
             if (q < J) *(float4 *)(rows + q * dq) = acc[q];
         if (d0 == 0) {
-            c.part_ml[j.dst_slot * 2 * kMaxGroup + g] = M;
-            c.part_ml[j.dst_slot * 2 * kMaxGroup + kMaxGroup + g] = L;
+            slot[g] = M;
+            slot[kMaxGroup + g] = L;
         }
         if (j.copy_base != 0) {
             const uint32_t crow = j.copy_base + (g * j.copy_pitch + d0) * 4;
@@ -1271,13 +1270,13 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     // memory) fetches the other CTAs' partials into its idle ring with bulk copies and folds them
     // with its own; a pair cut into more than kTreeFrom partials is folded in two levels.
     FoldCtx fc;
-    fc.part_acc = p.part_acc; fc.part_ml = p.part_ml; fc.status = p.status;
+    fc.part = p.part; fc.status = p.status;
     fc.ncols = ncols; fc.lane = lane;
     fc.fg = fold_geometry(ncols, D, lane);
     fc.out_off = (fc.fg.g / G) * qi_stride + (fc.fg.g % G) * D + fc.fg.d0;
     const uint32_t staging_u32 = smem_u32(smem + Lay::kStagingOff), park_u32 = smem_u32(smem + Lay::kParkOff);
     constexpr int kStagingMl = kMaxGroup * Lay::kStagePitch * 4, kParkMl = kMaxGroup * D * 4;
-    const int part_bytes = fc.fg.ncp * D * 4 + 64;               // a fetched partial in the ring: rows, then (m, l)
+    const int part_bytes = fc.fg.ncp * D * 4 + 64;               // a fetched partial in the ring: (m, l), then the live rows
     int bar_uses[2] = {(done + NS - 1) / NS, (done + NS - 2) / NS};   // phases the first two stage barriers have completed
     FoldJob jobs[2];
     int n_jobs = 0;
@@ -1287,7 +1286,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
     auto grid_job = [&](int c_first, int n, int i0, int istride, int alt_t, uint32_t buf, bool in_staging) {
         FoldJob j;
         j.n = n; j.cap = 1;                       // the ring region and cap are set when the jobs are started
-        j.base = 0; j.stride = part_bytes; j.pitch = D; j.ml_off = part_bytes - 64;
+        j.base = 0; j.stride = part_bytes; j.pitch = D; j.ml_off = -64;   // as fetched: (m, l), then the rows at `base`
         j.alt_t = alt_t; j.alt_base = buf;
         j.alt_pitch = in_staging ? Lay::kStagePitch : D; j.alt_ml_off = in_staging ? kStagingMl : kParkMl;
         j.fetch = 1; j.s_first = c_first; j.slot_first = 2 * c_first + 1; j.i0 = i0; j.istride = istride;
@@ -1401,7 +1400,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             // member, right away and with the whole ring; then count the group in
             FoldJob j = grid_job(tree_first[k], grp_cnt[k], grp[k] * sub[k], 1, me - grp[k] * sub[k], tree_buf[k], k == 1);
             j.dst_slot = j.slot_of(0);
-            j.base = ring; j.cap = min(32, NS * Lay::kStageBytes / part_bytes);
+            j.base = ring + 64; j.cap = min(32, NS * Lay::kStageBytes / part_bytes);
             j.bar = bars; j.uses = bar_uses[0];
             fence_proxy_async();                  // partials written through the generic proxy, read by bulk copies
             fold_fetch<D>(j, fc, 0);
@@ -1434,7 +1433,7 @@ paged_decode_attn_kernel(const __grid_constant__ CUtensorMap tmap, const AttnPar
             const int i = share ? (s & 1) : (s >> 1);
             const bool fetch = share ? s < 2 : !(s & 1);
             if (fetch) {
-                jobs[i].base = ring + (share ? i * (whole / 2) : 0);
+                jobs[i].base = ring + 64 + (share ? i * (whole / 2) : 0);
                 jobs[i].cap = min(32, (share ? whole / 2 : whole) / part_bytes);
                 jobs[i].bar = bars + i * 8;
                 jobs[i].uses = bar_uses[i];

@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel on the headline
 # workload, from the ncu capture summarised in profiles/paged_decode_attn_llama8b_b64.md.  Set to
 # None whenever the kernel changes after the capture.
-NCU_TRAFFIC_BYTES = 573.9e6    # dram read + write per launch of the attention kernel, mean of 2 captured launches (profiles/paged_decode_attn_llama8b_b64.md)
+NCU_TRAFFIC_BYTES = 573.6e6    # dram read + write per launch of the attention kernel, mean of 2 captured launches (profiles/paged_decode_attn_llama8b_b64.md)
 
 
 # ------------------------------------------------------------------------------- clocks

@@ -81,8 +81,10 @@ size_t kv_workspace_bytes(const ckv_config *cfg);
  * KV cache of Section 2.1 "PagedAttention").  d_pool must be 256-byte aligned and hold
  * kv_pool_bytes(); d_workspace must be 256-byte aligned and hold kv_workspace_bytes().  The
  * workspace is cleared on the default stream and the call synchronises once.  `device` is the
- * CUDA device ordinal both buffers live on.  Errors: CKV_EINVAL (shape, alignment),
- * CKV_ENOMEM (a size too small), CKV_ECUDA.
+ * CUDA device ordinal both buffers live on; the call makes it the calling thread's current
+ * device and leaves it so.  Every later call that takes the handle must be made with that device
+ * current and returns CKV_EINVAL otherwise (it would launch on the wrong GPU).  Errors:
+ * CKV_EINVAL (shape, alignment), CKV_ENOMEM (a size too small), CKV_ECUDA.
  */
 int32_t kv_pool_create(const ckv_config *cfg, void *d_pool, size_t pool_bytes,
                        void *d_workspace, size_t workspace_bytes, int32_t device,

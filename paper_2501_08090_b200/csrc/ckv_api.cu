@@ -196,12 +196,18 @@ int32_t launch_attention(ckv_pool *pool, const ckv::AttnParams &ap, cudaStream_t
     return CKV_OK;
 }
 
-int32_t check_call(ckv_pool *pool, int32_t layer, int32_t batch, const char *fn)
+int32_t check_device(const ckv_pool *pool, const char *fn)
 {
     if (!pool) return fail(CKV_EINVAL, "%s: pool is NULL", fn);
     int current = -1;
     if (cudaGetDevice(&current) != cudaSuccess || current != pool->device)
         return fail(CKV_EINVAL, "%s: the pool lives on device %d but device %d is current", fn, pool->device, current);
+    return CKV_OK;
+}
+
+int32_t check_call(ckv_pool *pool, int32_t layer, int32_t batch, const char *fn)
+{
+    if (int32_t rc = check_device(pool, fn)) return rc;
     if (layer < 0 || layer >= pool->cfg.num_layers)
         return fail(CKV_EINVAL, "%s: layer %d outside [0, %d)", fn, layer, pool->cfg.num_layers);
     if (batch < 1 || batch > pool->cfg.max_batch)
@@ -271,7 +277,11 @@ int32_t launch_read_probe(ckv_pool *pool, const ckv::ProbeParams &pp, cudaStream
 {
     using Lay = ckv::AttnLayout<D, W, NS>;
     auto kernel = ckv::pool_read_probe_kernel<D, W, NS>;
-    CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
+    static thread_local int configured_device = -1;
+    if (configured_device != pool->device) {
+        CKV_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay::kSmemBytes));
+        configured_device = pool->device;
+    }
     kernel<<<(pool->num_spans + W - 1) / W, W * 32, Lay::kSmemBytes, stream>>>(pool->tmap, pp);
     CKV_CUDA(cudaGetLastError());
     return CKV_OK;
@@ -490,9 +500,13 @@ static int32_t attention_launch(ckv_pool *pool, const char *fn, int32_t layer, i
     cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     if (pool->profile && pool->ev_used < kMaxProfile) {
         if ((size_t)(2 * pool->ev_used + 2) > pool->ev.size()) {
-            cudaEvent_t a, b;
+            cudaEvent_t a = nullptr, b = nullptr;
             CKV_CUDA(cudaEventCreate(&a));
-            CKV_CUDA(cudaEventCreate(&b));
+            const cudaError_t ce = cudaEventCreate(&b);
+            if (ce != cudaSuccess) {
+                cudaEventDestroy(a);
+                return fail(CKV_ECUDA, "%s: cudaEventCreate failed: %s", fn, cudaGetErrorString(ce));
+            }
             pool->ev.push_back(a);
             pool->ev.push_back(b);
         }
@@ -585,7 +599,7 @@ int32_t decode_plan(ckv_pool *pool, int32_t batch, const int32_t *d_seq_lens, vo
 
 int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits)
 {
-    if (!pool) return fail(CKV_EINVAL, "kv_check_status: pool is NULL");
+    if (int32_t rc = check_device(pool, "kv_check_status")) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint32_t bits = 0;
     CKV_CUDA(cudaMemcpyAsync(&bits, pool->d_ws + pool->ws.status, sizeof bits, cudaMemcpyDeviceToHost, s));
@@ -606,7 +620,7 @@ int32_t kv_check_status(ckv_pool *pool, void *stream, uint32_t *out_bits)
 
 int32_t ckv_wait_limit_selftest(ckv_pool *pool, uint64_t limit_ns, void *stream)
 {
-    if (!pool) return fail(CKV_EINVAL, "ckv_wait_limit_selftest: pool is NULL");
+    if (int32_t rc = check_device(pool, "ckv_wait_limit_selftest")) return rc;
     if (limit_ns < 1000 || limit_ns > 100000000ull)
         return fail(CKV_EINVAL, "ckv_wait_limit_selftest: limit outside [1 us, 100 ms]");
     ckv::wait_limit_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(
@@ -703,7 +717,7 @@ int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch
                            int32_t iters, void *d_flush, size_t flush_bytes, void *stream,
                            double *out_median_us, double *out_min_us)
 {
-    if (!pool) return fail(CKV_EINVAL, "step_latency_sweep: pool is NULL");
+    if (int32_t rc = check_device(pool, "step_latency_sweep")) return rc;
     if (n_sizes < 1 || !batch_sizes || !out_median_us || !out_min_us) return fail(CKV_EINVAL, "step_latency_sweep: bad size list or outputs");
     if (warmup < 0 || iters < 1 || iters > 100000) return fail(CKV_EINVAL, "step_latency_sweep: bad warmup/iters");
     if (batch_stride < 1 || batch_stride > pool->cfg.max_batch) return fail(CKV_EINVAL, "step_latency_sweep: bad batch_stride");
@@ -780,6 +794,7 @@ int32_t step_latency_sweep(ckv_pool *pool, int32_t n_sizes, const int32_t *batch
 int32_t ckv_read_span_trace(ckv_pool *pool, void *stream, uint64_t *h_trace, int32_t *h_span_start)
 {
     if (!pool || !h_trace) return fail(CKV_EINVAL, "ckv_read_span_trace: NULL argument");
+    if (int32_t rc = check_device(pool, "ckv_read_span_trace")) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     CKV_CUDA(cudaMemcpyAsync(h_trace, pool->d_ws + pool->ws.trace, sizeof(uint64_t) * 8 * pool->num_spans,
                              cudaMemcpyDeviceToHost, s));
@@ -908,7 +923,7 @@ int32_t decode_attention_noalloc(const ckv_config *cfg, const void *d_pool, int3
 static int32_t swap_launch(ckv_pool *pool, const char *fn, bool to_host, int32_t n_pages, const int32_t *d_page_ids,
                            void *h_image, size_t image_bytes, void *stream)
 {
-    if (!pool) return fail(CKV_EINVAL, "%s: pool is NULL", fn);
+    if (int32_t rc = check_device(pool, fn)) return rc;
     if (n_pages < 1 || !d_page_ids || !h_image) return fail(CKV_EINVAL, "%s: bad page list or image", fn);
     const ckv_config &c = pool->cfg;
     const size_t page_bytes = (size_t)c.num_kv_heads * 2 * c.page_size * c.head_dim * 2;

@@ -220,15 +220,31 @@ class KvPool:
         n = c.num_layers * c.num_pages * c.num_kv_heads * 2 * c.page_size * c.head_dim
         return self.pool.view(-1)[:n].view(c.num_layers, c.num_pages, c.num_kv_heads, 2, c.page_size, c.head_dim)
 
+    def _check_sizes(self, batch: int, block_tables, q_len: int = 1, q=None, kv=(), out=None) -> None:
+        """The C ABI takes bare pointers and cannot see a tensor that is too small or a table with
+        another row width; the device would read past it.  Checked here, where the sizes are known."""
+        c = self.cfg
+        if block_tables.numel() < batch * c.max_pages_per_req or \
+                (block_tables.dim() == 2 and block_tables.shape[1] != c.max_pages_per_req):
+            raise ValueError("block_tables must be [batch=%d][max_pages_per_req=%d], got %s"
+                             % (batch, c.max_pages_per_req, tuple(block_tables.shape)))
+        need_q = batch * q_len * c.num_q_heads * c.head_dim
+        need_kv = batch * q_len * c.num_kv_heads * c.head_dim
+        for name, t, need in [("q", q, need_q), ("out", out, need_q)] + [("k_new / v_new", t, need_kv) for t in kv]:
+            if t is not None and t.numel() < need:
+                raise ValueError("%s holds %d elements, %d needed for batch %d" % (name, t.numel(), need, batch))
+
     # -- the hot path
     def kv_append(self, layer: int, block_tables, seq_lens, k_new, v_new, stream=None) -> None:
         batch = int(seq_lens.shape[0])
+        self._check_sizes(batch, block_tables, kv=(k_new, v_new))
         _check(lib.kv_append(self._h, layer, batch, _dev_ptr(block_tables, torch.int32),
                              _dev_ptr(seq_lens, torch.int32), _dev_ptr(k_new, torch.bfloat16),
                              _dev_ptr(v_new, torch.bfloat16), _stream_ptr(stream)))
 
     def decode_attention(self, layer: int, block_tables, seq_lens, q, out, stream=None) -> None:
         batch = int(seq_lens.shape[0])
+        self._check_sizes(batch, block_tables, q=q, out=out)
         _check(lib.decode_attention(self._h, layer, batch, _dev_ptr(block_tables, torch.int32),
                                     _dev_ptr(seq_lens, torch.int32), _dev_ptr(q, torch.bfloat16),
                                     _dev_ptr(out, torch.bfloat16), _stream_ptr(stream)))
@@ -236,6 +252,7 @@ class KvPool:
     def decode_step(self, layer: int, block_tables, seq_lens, q, k_new, v_new, out, stream=None) -> None:
         """kv_append + decode_attention of one layer in a single kernel."""
         batch = int(seq_lens.shape[0])
+        self._check_sizes(batch, block_tables, q=q, kv=(k_new, v_new), out=out)
         _check(lib.decode_step(self._h, layer, batch, _dev_ptr(block_tables, torch.int32),
                                _dev_ptr(seq_lens, torch.int32), _dev_ptr(q, torch.bfloat16),
                                _dev_ptr(k_new, torch.bfloat16), _dev_ptr(v_new, torch.bfloat16),
@@ -243,12 +260,14 @@ class KvPool:
 
     def kv_append_multi(self, layer: int, q_len: int, block_tables, seq_lens, k_new, v_new, stream=None) -> None:
         """Append q_len new tokens per request (k_new, v_new [batch][q_len][Hkv][d])."""
+        self._check_sizes(int(seq_lens.shape[0]), block_tables, q_len=int(q_len), kv=(k_new, v_new))
         _check(lib.kv_append_multi(self._h, layer, int(seq_lens.shape[0]), int(q_len),
                                    _dev_ptr(block_tables, torch.int32), _dev_ptr(seq_lens, torch.int32),
                                    _dev_ptr(k_new, torch.bfloat16), _dev_ptr(v_new, torch.bfloat16), _stream_ptr(stream)))
 
     def decode_attention_multi(self, layer: int, q_len: int, block_tables, seq_lens, q, out, stream=None) -> None:
         """Causal attention of the q_len new tokens (q, out [batch][q_len][Hq][d])."""
+        self._check_sizes(int(seq_lens.shape[0]), block_tables, q_len=int(q_len), q=q, out=out)
         _check(lib.decode_attention_multi(self._h, layer, int(seq_lens.shape[0]), int(q_len),
                                           _dev_ptr(block_tables, torch.int32), _dev_ptr(seq_lens, torch.int32),
                                           _dev_ptr(q, torch.bfloat16), _dev_ptr(out, torch.bfloat16), _stream_ptr(stream)))
@@ -273,6 +292,7 @@ class KvPool:
 
     def read_probe(self, layer: int, block_tables, seq_lens, stream=None) -> None:
         """Stream the KV tiles decode_attention would read for this batch, without the arithmetic."""
+        self._check_sizes(int(seq_lens.shape[0]), block_tables)
         _check(lib.kv_read_probe(self._h, layer, int(seq_lens.shape[0]), _dev_ptr(block_tables, torch.int32),
                                  _dev_ptr(seq_lens, torch.int32), _stream_ptr(stream)))
 
@@ -312,6 +332,7 @@ class KvPool:
             if t.is_cuda or not t.is_contiguous():
                 raise ValueError("decode_step_host takes contiguous host tensors")
         batch = int(seq_lens.shape[0])
+        self._check_sizes(batch, block_tables, q=q, kv=(k_new, v_new), out=out)
         _check(lib.decode_step_host(self._h, layer, batch, block_tables.data_ptr(), seq_lens.data_ptr(),
                                     q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(),
                                     _stream_ptr(stream)))
@@ -326,6 +347,7 @@ class KvPool:
         for t in (block_tables, seq_lens, q, k_new, v_new, out):
             if t.is_cuda or not t.is_contiguous():
                 raise ValueError("decode_step_host takes contiguous host tensors")
+        self._check_sizes(int(seq_lens.shape[0]), block_tables, q=q, kv=(k_new, v_new), out=out)
         keep = (block_tables, seq_lens, q, k_new, v_new, out)
         args = (self._h, int(layer), int(seq_lens.shape[0]), block_tables.data_ptr(), seq_lens.data_ptr(),
                 q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(), out.data_ptr(), _stream_ptr(stream))

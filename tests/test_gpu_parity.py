@@ -522,6 +522,23 @@ def test_arguments_are_validated_on_the_host():
         ds.pool.set_partition(0)
     with pytest.raises(b.CkvError):
         ds.pool.set_partition(3000)
-    big = torch.zeros(9, dtype=torch.int32, device="cuda")
-    with pytest.raises(b.CkvError):
-        ds.pool.decode_attention(0, ds.bt, big, ds.q[0], ds.out[0])          # batch > max_batch
+    big = torch.ones(9, dtype=torch.int32, device="cuda")
+    big_bt = torch.zeros((9, ds.bt.shape[1]), dtype=torch.int32, device="cuda")
+    big_q = torch.zeros((9,) + tuple(ds.q[0].shape[1:]), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(b.CkvError) as e:
+        ds.pool.decode_attention(0, big_bt, big, big_q, torch.zeros_like(big_q))   # batch > max_batch
+    assert e.value.code == b.CKV_EINVAL
+    # tensors too small for the batch, or a table with another row width, never reach the device
+    with pytest.raises(ValueError):
+        ds.pool.decode_attention(0, ds.bt, big, ds.q[0], ds.out[0])
+    with pytest.raises(ValueError):
+        ds.pool.decode_attention(0, ds.bt[:, :-1].contiguous(), ds.sl, ds.q[0], ds.out[0])
+    with pytest.raises(ValueError):
+        ds.pool.decode_step(0, ds.bt, ds.sl, ds.q[0], ds.k_new[0][:-1], ds.v_new[0], ds.out[0])
+    with pytest.raises(ValueError):
+        ds.pool.decode_step(0, ds.bt, ds.sl, ds.q[0][:-1], ds.k_new[0], ds.v_new[0], ds.out[0])
+    with pytest.raises(ValueError):
+        ds.pool.kv_append(0, ds.bt, ds.sl, ds.k_new[0], ds.v_new[0][:-1])
+    # and nothing above disturbed the pool: a regular step still matches
+    ds.pool.decode_step(0, ds.bt, ds.sl, ds.q[0], ds.k_new[0], ds.v_new[0], ds.out[0])
+    assert ds.pool.check_status() == 0

@@ -367,6 +367,13 @@ class KvPool:
         med = np.zeros(sizes.size, dtype=np.float64)
         mn = np.zeros(sizes.size, dtype=np.float64)
         stride = int(seq_lens.shape[0])
+        self._check_sizes(stride, block_tables)
+        c = self.cfg                                   # q, k_new, v_new, out: [layers][stride][heads][d]
+        for name, t, heads in (("q", q, c.num_q_heads), ("out", out, c.num_q_heads),
+                               ("k_new", k_new, c.num_kv_heads), ("v_new", v_new, c.num_kv_heads)):
+            if t.numel() < c.num_layers * stride * heads * c.head_dim:
+                raise ValueError("%s holds %d elements, %d needed for %d layers of batch %d"
+                                 % (name, t.numel(), c.num_layers * stride * heads * c.head_dim, c.num_layers, stride))
         fl_ptr = _dev_ptr(flush) if flush is not None else None
         fl_bytes = flush.numel() * flush.element_size() if flush is not None else 0
         _check(lib.step_latency_sweep(self._h, int(sizes.size), sizes.ctypes.data, stride,
@@ -404,6 +411,15 @@ def decode_attention_noalloc(cfg: Config, pool: torch.Tensor, layer: int, block_
     """decode_attention for callers that cannot allocate a workspace: partial results go into a fixed
     array inside the library (at most 640 spans).  Runs on the current CUDA device.  With `sync`
     the stream is synchronised and the device status bits are returned (and raised if non-zero)."""
+    batch = int(seq_lens.shape[0])
+    if block_tables.numel() < batch * cfg.max_pages_per_req or \
+            (block_tables.dim() == 2 and block_tables.shape[1] != cfg.max_pages_per_req):
+        raise ValueError("block_tables must be [batch=%d][max_pages_per_req=%d], got %s"
+                         % (batch, cfg.max_pages_per_req, tuple(block_tables.shape)))
+    if min(q.numel(), out.numel()) < batch * cfg.num_q_heads * cfg.head_dim:
+        raise ValueError("q / out too small for batch %d" % batch)
+    if pool.numel() * pool.element_size() < kv_pool_bytes(cfg):
+        raise ValueError("pool tensor smaller than kv_pool_bytes(cfg)")
     bits = ctypes.c_uint32(0)
     rc = lib.decode_attention_noalloc(ctypes.byref(cfg), _dev_ptr(pool), int(layer), int(seq_lens.shape[0]),
                                       _dev_ptr(block_tables, torch.int32), _dev_ptr(seq_lens, torch.int32),

@@ -144,4 +144,14 @@ def test_fused_loop_at_full_size_with_poisoned_future_slots():
         ref = oracle.decode_attention(ref_pool, sh, 0, bt, lens, q_h[s])
         assert_close(got[s], ref, "step %d" % s)
     assert np.array_equal(dev_to_bits(kp.pool), ref_pool)
+
+    # the same loop in plain stream order (no launch overlaps its predecessor): same bits
+    kp.pool.copy_(bits_to_dev(pool_h))
+    kp.set_overlap(False)
+    out2 = torch.full_like(q, float("nan"))
+    for s in range(steps):
+        kp.decode_step(0, btd, lens_d[s], q[s], k[s], v[s], out2[s])
+    assert kp.check_status() == 0
+    assert np.array_equal(dev_to_bits(out2), got)
+    assert np.array_equal(dev_to_bits(kp.pool), ref_pool)
     kp.close()
